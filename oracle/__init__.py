@@ -1,0 +1,254 @@
+"""Few-Bit Backward reference oracle -- TEST INFRASTRUCTURE, not the product.
+
+A ctypes view of ``fewbit_oracle.c`` (plain C, binary64 arithmetic, written
+from the paper).  Only the tests, the smoke check and the benchmark's CPU
+baseline may import this package; the CUDA library never does and shares no
+code with it.
+
+The shared object is compiled with ``gcc -O2 -ffp-contract=off`` (no fused
+multiply-add contraction, no fast-math) the first time it is needed.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fewbit_oracle.c")
+_LIB = os.path.join(_HERE, "libfewbit_oracle.so")
+
+ACTS = {
+    "gelu": 0, "silu": 1, "sigmoid": 2, "tanh": 3, "elu": 4, "softplus": 5,
+    "leaky_relu": 6, "relu": 7, "selu": 8,
+}
+
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc; returns the path of the shared object."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call([
+            "gcc", "-std=c11", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
+            "-D_GNU_SOURCE", "-o", tmp, _SRC, "-lm",
+        ])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is not None:
+            return _lib
+        lib = ctypes.CDLL(build())
+        c_dp = ctypes.POINTER(ctypes.c_double)
+        c_ip = ctypes.POINTER(ctypes.c_int)
+        vp = ctypes.c_void_p
+        sz = ctypes.c_size_t
+        lib.fbo_act.restype = ctypes.c_double
+        lib.fbo_act.argtypes = [ctypes.c_int, ctypes.c_double]
+        lib.fbo_act_deriv.restype = ctypes.c_double
+        lib.fbo_act_deriv.argtypes = [ctypes.c_int, ctypes.c_double]
+        lib.fbo_dp_solve.restype = ctypes.c_int
+        lib.fbo_dp_solve.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_int,
+                                     ctypes.c_int, c_dp, c_dp, c_dp, c_ip]
+        lib.fbo_objective.restype = ctypes.c_int
+        lib.fbo_objective.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_int,
+                                      ctypes.c_int, c_ip, c_dp]
+        lib.fbo_bruteforce.restype = ctypes.c_int
+        lib.fbo_bruteforce.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_int,
+                                       ctypes.c_int, c_ip, c_dp]
+        lib.fbo_packed_words.restype = sz
+        lib.fbo_packed_words.argtypes = [sz, ctypes.c_int]
+        lib.fbo_pack.restype = None
+        lib.fbo_pack.argtypes = [ctypes.c_int, vp, vp, sz]
+        lib.fbo_unpack.restype = None
+        lib.fbo_unpack.argtypes = [ctypes.c_int, vp, vp, sz]
+        for name in ("fbo_fwd_f32", "fbo_fwd_bf16"):
+            fn = getattr(lib, name)
+            fn.restype = None
+            fn.argtypes = [ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, sz]
+        for name in ("fbo_bwd_f32", "fbo_bwd_bf16"):
+            fn = getattr(lib, name)
+            fn.restype = None
+            fn.argtypes = [ctypes.c_int, vp, vp, vp, vp, sz]
+        for name in ("fbo_act_array", "fbo_act_deriv_array"):
+            fn = getattr(lib, name)
+            fn.restype = None
+            fn.argtypes = [ctypes.c_int, vp, vp, sz]
+        lib.fbo_f64_to_bf16_array.restype = None
+        lib.fbo_f64_to_bf16_array.argtypes = [vp, vp, sz]
+        _lib = lib
+        return lib
+
+
+def _act_id(act) -> int:
+    return ACTS[act] if isinstance(act, str) else int(act)
+
+
+def _ptr(a: np.ndarray):
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+# ----------------------------------------------------------------------------
+# activations (binary64)
+# ----------------------------------------------------------------------------
+def act(name, x) -> np.ndarray:
+    """f(x) in binary64 (Sec. 2)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    y = np.empty_like(x)
+    _load().fbo_act_array(_act_id(name), _ptr(x), _ptr(y), x.size)
+    return y
+
+
+def act_deriv(name, x) -> np.ndarray:
+    """f'(x) in binary64 (Eq. 1)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    y = np.empty_like(x)
+    _load().fbo_act_deriv_array(_act_id(name), _ptr(x), _ptr(y), x.size)
+    return y
+
+
+def f64_to_bf16(x) -> np.ndarray:
+    """binary64 -> bfloat16 bit patterns (uint16), one round-to-nearest-even."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    y = np.empty(x.shape, dtype=np.uint16)
+    _load().fbo_f64_to_bf16_array(_ptr(x), _ptr(y), x.size)
+    return y
+
+
+def bf16_to_f64(h) -> np.ndarray:
+    h = np.ascontiguousarray(h, dtype=np.uint16)
+    return (h.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+# ----------------------------------------------------------------------------
+# tables (Eq. 3, 4, 7-9)
+# ----------------------------------------------------------------------------
+def dp_solve(name, bits=None, A=-8.0, B=8.0, n_cells=4096, K=None):
+    """Optimal K-piece constant approximation of f' on the grid (Eq. 7).
+
+    Returns a dict with ``s`` (K-1 boundaries, f64), ``lev`` (K levels, f64),
+    ``idx`` (grid indices of the boundaries) and ``objective`` (Eq. 3)."""
+    if K is None:
+        K = 1 << int(bits)
+    s = np.zeros(max(K - 1, 1), dtype=np.float64)
+    lev = np.zeros(K, dtype=np.float64)
+    idx = np.zeros(max(K - 1, 1), dtype=np.int32)
+    obj = ctypes.c_double(0.0)
+    rc = _load().fbo_dp_solve(
+        _act_id(name), float(A), float(B), int(n_cells), int(K),
+        s.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
+        lev.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
+        ctypes.byref(obj),
+        idx.ctypes.data_as(ctypes.POINTER(ctypes.c_int)))
+    if rc != 0:
+        raise ValueError(f"fbo_dp_solve failed with {rc}")
+    return {"s": s[:K - 1].copy(), "lev": lev, "idx": idx[:K - 1].copy(), "objective": obj.value}
+
+
+def objective(name, idx, A, B, n_cells) -> float:
+    """Eq. 3 for boundaries at the grid indices ``idx`` (levels by Eq. 4)."""
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    K = idx.size + 1
+    obj = ctypes.c_double(0.0)
+    rc = _load().fbo_objective(_act_id(name), float(A), float(B), int(n_cells), K,
+                               idx.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), ctypes.byref(obj))
+    if rc != 0:
+        raise ValueError(f"fbo_objective failed with {rc}")
+    return obj.value
+
+
+def bruteforce(name, K, A, B, n_cells):
+    """Exhaustive minimiser of Eq. 3 over all boundary subsets of the grid."""
+    idx = np.zeros(max(K - 1, 1), dtype=np.int32)
+    obj = ctypes.c_double(0.0)
+    rc = _load().fbo_bruteforce(_act_id(name), float(A), float(B), int(n_cells), int(K),
+                                idx.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), ctypes.byref(obj))
+    if rc != 0:
+        raise ValueError(f"fbo_bruteforce failed with {rc}")
+    return {"idx": idx[:K - 1].copy(), "objective": obj.value}
+
+
+# ----------------------------------------------------------------------------
+# bit stream
+# ----------------------------------------------------------------------------
+def packed_words(n: int, bits: int) -> int:
+    return (int(n) * int(bits) + 31) // 32
+
+
+def pack(codes, bits: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.zeros(packed_words(codes.size, bits), dtype=np.uint32)
+    _load().fbo_pack(int(bits), _ptr(codes), _ptr(out), codes.size)
+    return out
+
+
+def unpack(packed, bits: int, n: int) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint32)
+    assert packed.size >= packed_words(n, bits)
+    out = np.zeros(n, dtype=np.uint8)
+    _load().fbo_unpack(int(bits), _ptr(packed), _ptr(out), n)
+    return out
+
+
+# ----------------------------------------------------------------------------
+# hot path (Listing 1)
+# ----------------------------------------------------------------------------
+def _check_tables(bits, s=None, lev=None):
+    K = 1 << int(bits)
+    if s is not None:
+        s = np.ascontiguousarray(s, dtype=np.float32)
+        assert s.size == K - 1
+    if lev is not None:
+        lev = np.ascontiguousarray(lev, dtype=np.float32)
+        assert lev.size == K
+    return s, lev
+
+
+def fwd(name, bits: int, s, x: np.ndarray):
+    """Forward half: returns (y, packed).
+
+    ``x`` is float32, or uint16 holding bfloat16 bit patterns; ``y`` has the
+    same dtype.  ``s`` are the K-1 boundaries as binary32."""
+    s, _ = _check_tables(bits, s=s)
+    if s.size == 0:
+        s = np.zeros(1, dtype=np.float32)
+    x = np.ascontiguousarray(x)
+    n = x.size
+    packed = np.zeros(packed_words(n, bits), dtype=np.uint32)
+    y = np.empty_like(x)
+    lib = _load()
+    if x.dtype == np.float32:
+        lib.fbo_fwd_f32(_act_id(name), int(bits), _ptr(s), _ptr(x), _ptr(y), _ptr(packed), n)
+    elif x.dtype == np.uint16:
+        lib.fbo_fwd_bf16(_act_id(name), int(bits), _ptr(s), _ptr(x), _ptr(y), _ptr(packed), n)
+    else:
+        raise TypeError("x must be float32 or uint16 (bfloat16 bits)")
+    return y, packed
+
+
+def bwd(bits: int, lev, packed: np.ndarray, grad_out: np.ndarray, n: int | None = None):
+    """Backward half: returns grad_in (same dtype convention as ``fwd``)."""
+    _, lev = _check_tables(bits, lev=lev)
+    grad_out = np.ascontiguousarray(grad_out)
+    packed = np.ascontiguousarray(packed, dtype=np.uint32)
+    if n is None:
+        n = grad_out.size
+    assert packed.size >= packed_words(n, bits)
+    grad_in = np.empty_like(grad_out)
+    lib = _load()
+    if grad_out.dtype == np.float32:
+        lib.fbo_bwd_f32(int(bits), _ptr(lev), _ptr(packed), _ptr(grad_out), _ptr(grad_in), n)
+    elif grad_out.dtype == np.uint16:
+        lib.fbo_bwd_bf16(int(bits), _ptr(lev), _ptr(packed), _ptr(grad_out), _ptr(grad_in), n)
+    else:
+        raise TypeError("grad_out must be float32 or uint16 (bfloat16 bits)")
+    return grad_in

@@ -1,0 +1,411 @@
+/*
+ * Few-Bit Backward -- reference oracle (TEST INFRASTRUCTURE, not the product).
+ *
+ * A plain, slow, single-threaded CPU statement of what the hot path computes,
+ * written from the paper (arXiv 2202.00441) so that a reader can check it
+ * against the equations by eye.  It shares no code with the CUDA library and
+ * is only ever called from tests, the smoke check and the benchmark's CPU
+ * baseline.  Everything floating point is binary64 unless the contract fixes
+ * a narrower type (the fp32 compare in the bucketize step and the fp32
+ * multiply in the backward step).
+ *
+ * Parts and the passage each follows:
+ *   fbo_act / fbo_act_deriv   Sec. 2 (pointwise f, chain rule Eq. 1); the
+ *                             activations of Table 1 plus ELU / LeakyReLU
+ *   fbo_dp_solve              Eq. 7 (discrete DP, k-1 on the right-hand side as
+ *                             in Eq. 6), Eq. 8-9 (prefix integrals), Eq. 4
+ *                             (optimal levels), uniform weight Eq. 10
+ *   fbo_bruteforce            Eq. 3 minimised by exhaustive search on the grid
+ *   fbo_objective             Eq. 3 for a given boundary set (levels by Eq. 4)
+ *   fbo_fwd_*                 Listing 1 "forward": y = f(x); code = position
+ *                             of x among the boundaries s (Eq. 2); only
+ *                             log2(K) bits per element are kept (Sec. 2)
+ *   fbo_bwd_*                 Listing 1 "backward": grad_in = grad_out * y[code]
+ *
+ * Every function here is pinned by tests/test_oracle_*.py against Table 1,
+ * brute force, closed forms and library routines; none is "parity unpinned"
+ * except the boundary indices of degenerate (piecewise-constant f') tables,
+ * where every zero-error table is equally correct.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum {
+    FBO_GELU = 0,      /* x * Phi(x), erf form */
+    FBO_SILU = 1,      /* x * sigmoid(x) (Swish) */
+    FBO_SIGMOID = 2,
+    FBO_TANH = 3,
+    FBO_ELU = 4,       /* alpha = 1 */
+    FBO_SOFTPLUS = 5,  /* beta = 1, no threshold */
+    FBO_LEAKY_RELU = 6,/* slope 0.01 */
+    FBO_RELU = 7,      /* Table 1 row, pin only */
+    FBO_SELU = 8       /* Table 1 row, pin only */
+};
+
+#define SELU_LAMBDA 1.0507009873554804934193349852946
+#define SELU_ALPHA  1.6732632423543772848170429916717
+
+static double sigmoid64(double x)
+{
+    /* 1/(1+e^-x), written so that neither branch overflows */
+    if (x >= 0.0) return 1.0 / (1.0 + exp(-x));
+    double e = exp(x);
+    return e / (1.0 + e);
+}
+
+static double std_normal_cdf(double x) { return 0.5 * erfc(-x * M_SQRT1_2); }
+static double std_normal_pdf(double x) { return exp(-0.5 * x * x) / sqrt(2.0 * M_PI); }
+
+/* f(x), Sec. 2. */
+double fbo_act(int act, double x)
+{
+    switch (act) {
+    case FBO_GELU:       return x * std_normal_cdf(x);
+    case FBO_SILU:       return x * sigmoid64(x);
+    case FBO_SIGMOID:    return sigmoid64(x);
+    case FBO_TANH:       return tanh(x);
+    case FBO_ELU:        return x > 0.0 ? x : expm1(x);
+    case FBO_SOFTPLUS:   return (x > 0.0 ? x : 0.0) + log1p(exp(-fabs(x)));
+    case FBO_LEAKY_RELU: return x > 0.0 ? x : 0.01 * x;
+    case FBO_RELU:       return x > 0.0 ? x : 0.0;
+    case FBO_SELU:       return SELU_LAMBDA * (x > 0.0 ? x : SELU_ALPHA * expm1(x));
+    default:             return NAN;
+    }
+}
+
+/* f'(x), the factor of the chain rule, Eq. 1. */
+double fbo_act_deriv(int act, double x)
+{
+    double s;
+    switch (act) {
+    case FBO_GELU:       return std_normal_cdf(x) + x * std_normal_pdf(x);
+    case FBO_SILU:       s = sigmoid64(x); return s * (1.0 + x * (1.0 - s));
+    case FBO_SIGMOID:    s = sigmoid64(x); return s * (1.0 - s);
+    case FBO_TANH:       s = tanh(x); return 1.0 - s * s;
+    case FBO_ELU:        return x > 0.0 ? 1.0 : exp(x);
+    case FBO_SOFTPLUS:   return sigmoid64(x);
+    case FBO_LEAKY_RELU: return x > 0.0 ? 1.0 : 0.01;
+    case FBO_RELU:       return x > 0.0 ? 1.0 : 0.0;
+    case FBO_SELU:       return SELU_LAMBDA * (x > 0.0 ? 1.0 : SELU_ALPHA * exp(x));
+    default:             return NAN;
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Prefix integrals of Eq. 8-9 with the uniform weight of Eq. 10 on [A,B].   */
+/*   W(i)  = t_i - A                       (integral of w)                   */
+/*   FW(i) = f(t_i) - f(A)                 (integral of f' w, closed form)   */
+/*   F2(i) = F2(i-1) + int_cell f'^2       (4-point Gauss-Legendre per cell; */
+/*           the nodes are interior, so a jump of f' at a grid point is      */
+/*           never sampled)                                                  */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+    int n;
+    double *t, *W, *FW, *F2;
+} prefix_t;
+
+static int prefix_build(prefix_t *p, int act, double A, double B, int n)
+{
+    static const double gl_x[4] = { -0.86113631159405257522, -0.33998104358485626480,
+                                     0.33998104358485626480,  0.86113631159405257522 };
+    static const double gl_w[4] = {  0.34785484513745385737,  0.65214515486254614263,
+                                     0.65214515486254614263,  0.34785484513745385737 };
+    p->n = n;
+    p->t  = (double *)malloc(sizeof(double) * (size_t)(n + 1));
+    p->W  = (double *)malloc(sizeof(double) * (size_t)(n + 1));
+    p->FW = (double *)malloc(sizeof(double) * (size_t)(n + 1));
+    p->F2 = (double *)malloc(sizeof(double) * (size_t)(n + 1));
+    if (!p->t || !p->W || !p->FW || !p->F2) return -1;
+    double fA = fbo_act(act, A);
+    for (int i = 0; i <= n; ++i) {
+        p->t[i]  = A + (B - A) * (double)i / (double)n;
+        p->W[i]  = p->t[i] - A;
+        p->FW[i] = fbo_act(act, p->t[i]) - fA;
+    }
+    p->t[n] = B;
+    p->F2[0] = 0.0;
+    for (int i = 0; i < n; ++i) {
+        double a = p->t[i], b = p->t[i + 1];
+        double mid = 0.5 * (a + b), half = 0.5 * (b - a), acc = 0.0;
+        for (int q = 0; q < 4; ++q) {
+            double d = fbo_act_deriv(act, mid + half * gl_x[q]);
+            acc += gl_w[q] * d * d;
+        }
+        p->F2[i + 1] = p->F2[i] + half * acc;
+    }
+    return 0;
+}
+
+static void prefix_free(prefix_t *p)
+{
+    free(p->t); free(p->W); free(p->FW); free(p->F2);
+}
+
+/* y(j,i) of Eq. 8: the optimal level (Eq. 4) of the bin [t_j, t_i]. */
+static double bin_level(const prefix_t *p, int j, int i)
+{
+    return (p->FW[i] - p->FW[j]) / (p->W[i] - p->W[j]);
+}
+
+/* T(j,i) of Eq. 8: the error of the bin [t_j, t_i] under its optimal level.
+ * It is a sum of squares, so a negative value can only be rounding noise and
+ * is clamped to zero. */
+static double bin_cost(const prefix_t *p, int j, int i)
+{
+    double y = bin_level(p, j, i);
+    double c = p->F2[i] - p->F2[j] - y * y * (p->W[i] - p->W[j]);
+    return c > 0.0 ? c : 0.0;
+}
+
+/*
+ * Discrete dynamic programme, Eq. 7:
+ *     DP(i,k) = min_j DP(j,k-1) + T(j,i),   DP(0,0) = 0,
+ * i = grid index of the right end, k = number of constant pieces used on
+ * [A, t_i].  The answer is DP(n,K); the first minimiser wins a tie.
+ * Outputs: idx_out[K-1] interior boundary grid indices (increasing),
+ * s_out[K-1] = t[idx], lev_out[K] by Eq. 4 with s_0 = A and s_K = B,
+ * *objective = DP(n,K).  Returns 0 on success.
+ */
+int fbo_dp_solve(int act, double A, double B, int n, int K,
+                 double *s_out, double *lev_out, double *objective, int *idx_out)
+{
+    if (n < 1 || K < 1 || K > n || !(A < B)) return -1;
+    prefix_t p;
+    if (prefix_build(&p, act, A, B, n)) return -2;
+    size_t stride = (size_t)(n + 1);
+    double *dp  = (double *)malloc(sizeof(double) * stride * (size_t)(K + 1));
+    int    *arg = (int *)malloc(sizeof(int) * stride * (size_t)(K + 1));
+    if (!dp || !arg) return -2;
+    for (size_t q = 0; q < stride * (size_t)(K + 1); ++q) { dp[q] = INFINITY; arg[q] = -1; }
+    dp[0] = 0.0; /* DP(0,0) */
+    for (int k = 1; k <= K; ++k) {
+        for (int i = k; i <= n; ++i) {
+            double best = INFINITY; int bestj = -1;
+            for (int j = k - 1; j < i; ++j) {
+                double prev = dp[(size_t)(k - 1) * stride + (size_t)j];
+                if (prev == INFINITY) continue;
+                double v = prev + bin_cost(&p, j, i);
+                if (v < best) { best = v; bestj = j; }
+            }
+            dp[(size_t)k * stride + (size_t)i] = best;
+            arg[(size_t)k * stride + (size_t)i] = bestj;
+        }
+    }
+    if (objective) *objective = dp[(size_t)K * stride + (size_t)n];
+    /* back-track the right ends of pieces K, K-1, ..., 1 */
+    int *ends = (int *)malloc(sizeof(int) * (size_t)(K + 1));
+    ends[K] = n;
+    for (int k = K; k >= 1; --k) ends[k - 1] = arg[(size_t)k * stride + (size_t)ends[k]];
+    /* ends[0] == 0 by construction */
+    for (int m = 1; m < K; ++m) {
+        if (idx_out) idx_out[m - 1] = ends[m];
+        if (s_out)   s_out[m - 1] = p.t[ends[m]];
+    }
+    if (lev_out)
+        for (int m = 0; m < K; ++m) lev_out[m] = bin_level(&p, ends[m], ends[m + 1]);
+    free(ends); free(dp); free(arg);
+    prefix_free(&p);
+    return 0;
+}
+
+/* Eq. 3 for the boundary grid indices idx[0..K-2] (levels by Eq. 4). */
+int fbo_objective(int act, double A, double B, int n, int K, const int *idx, double *objective)
+{
+    prefix_t p;
+    if (prefix_build(&p, act, A, B, n)) return -2;
+    double total = 0.0;
+    int left = 0;
+    for (int m = 0; m < K; ++m) {
+        int right = (m == K - 1) ? n : idx[m];
+        if (right <= left) { prefix_free(&p); return -1; }
+        total += bin_cost(&p, left, right);
+        left = right;
+    }
+    *objective = total;
+    prefix_free(&p);
+    return 0;
+}
+
+/*
+ * Exhaustive search: every increasing (K-1)-subset of the interior grid
+ * points 1..n-1, each scored by Eq. 3 with the levels of Eq. 4.  The
+ * lexicographically first minimiser is kept.  Only for tiny n.
+ */
+int fbo_bruteforce(int act, double A, double B, int n, int K, int *idx_out, double *objective)
+{
+    if (K < 1 || K > n) return -1;
+    prefix_t p;
+    if (prefix_build(&p, act, A, B, n)) return -2;
+    int m = K - 1;
+    int *c = (int *)malloc(sizeof(int) * (size_t)(m + 1));
+    for (int q = 0; q < m; ++q) c[q] = q + 1;
+    double best = INFINITY;
+    for (;;) {
+        double total = 0.0;
+        int left = 0;
+        for (int q = 0; q <= m; ++q) {
+            int right = (q == m) ? n : c[q];
+            total += bin_cost(&p, left, right);
+            left = right;
+        }
+        if (total < best) {
+            best = total;
+            for (int q = 0; q < m; ++q) idx_out[q] = c[q];
+        }
+        /* next combination of {1..n-1} choose m */
+        int q = m - 1;
+        while (q >= 0 && c[q] == (n - 1) - (m - 1 - q)) --q;
+        if (q < 0) break;
+        ++c[q];
+        for (int r = q + 1; r < m; ++r) c[r] = c[r - 1] + 1;
+    }
+    *objective = best;
+    free(c);
+    prefix_free(&p);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Rounding binary64 -> storage dtype, round-to-nearest-even, in ONE step.   */
+/* ------------------------------------------------------------------------ */
+
+/* bfloat16: 8 exponent bits, 7 stored mantissa bits.  The value is scaled so
+ * that one bfloat16 ulp becomes 1.0, rounded with nearbyint (nearest-even in
+ * the default rounding mode) and scaled back; both scalings are exact. */
+uint16_t fbo_f64_to_bf16(double d)
+{
+    if (isnan(d)) return 0x7fc0;
+    if (isinf(d)) return d > 0 ? 0x7f80 : 0xff80;
+    double r = 0.0;
+    if (d != 0.0) {
+        int e = ilogb(d);
+        if (e < -126) e = -126;           /* subnormal range: fixed spacing 2^-133 */
+        double ulp = ldexp(1.0, e - 7);
+        r = nearbyint(d / ulp) * ulp;
+    } else {
+        r = d;                             /* keeps the sign of zero */
+    }
+    float f = (float)r;                    /* exact, or +-inf past the largest finite bf16 */
+    if (fabs(r) >= ldexp(1.0, 128)) f = r > 0 ? INFINITY : -INFINITY;
+    uint32_t u; memcpy(&u, &f, 4);
+    if (r == 0.0 && signbit(d)) u = 0x80000000u;
+    return (uint16_t)(u >> 16);
+}
+
+double fbo_bf16_to_f64(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16; float f; memcpy(&f, &u, 4); return (double)f;
+}
+
+static float bf16_to_f32(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16; float f; memcpy(&f, &u, 4); return f;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Forward, Listing 1: y = f(x); X_pos = position of x among s; save X_pos   */
+/* in log2(K) bits.  Position = number of boundaries strictly below x, so    */
+/* bin i is (s_i, s_{i+1}] and values outside [A,B] fall in the end bins.    */
+/* Bit layout of the saved tensor: one flat bit stream, element e occupies   */
+/* bits [e*bits, e*bits+bits), least significant bit first, stored in        */
+/* little-endian 32-bit words; unused bits of the last word are zero.        */
+/* ------------------------------------------------------------------------ */
+static uint32_t bucketize(const float *s, int nb, float x)
+{
+    uint32_t c = 0;
+    for (int j = 0; j < nb; ++j) if (s[j] < x) ++c;
+    return c;
+}
+
+static void put_code(uint32_t *packed, size_t e, int bits, uint32_t code)
+{
+    for (int b = 0; b < bits; ++b) {
+        size_t pos = e * (size_t)bits + (size_t)b;
+        if ((code >> b) & 1u) packed[pos >> 5] |= (uint32_t)1 << (pos & 31);
+    }
+}
+
+static uint32_t get_code(const uint32_t *packed, size_t e, int bits)
+{
+    uint32_t code = 0;
+    for (int b = 0; b < bits; ++b) {
+        size_t pos = e * (size_t)bits + (size_t)b;
+        code |= ((packed[pos >> 5] >> (pos & 31)) & 1u) << b;
+    }
+    return code;
+}
+
+size_t fbo_packed_words(size_t n, int bits) { return (n * (size_t)bits + 31) / 32; }
+
+void fbo_pack(int bits, const uint8_t *codes, uint32_t *packed, size_t n)
+{
+    memset(packed, 0, 4 * fbo_packed_words(n, bits));
+    for (size_t e = 0; e < n; ++e) put_code(packed, e, bits, codes[e]);
+}
+
+void fbo_unpack(int bits, const uint32_t *packed, uint8_t *codes, size_t n)
+{
+    for (size_t e = 0; e < n; ++e) codes[e] = (uint8_t)get_code(packed, e, bits);
+}
+
+void fbo_fwd_f32(int act, int bits, const float *s, const float *x, float *y,
+                 uint32_t *packed, size_t n)
+{
+    int nb = (1 << bits) - 1;
+    memset(packed, 0, 4 * fbo_packed_words(n, bits));
+    for (size_t e = 0; e < n; ++e) {
+        y[e] = (float)fbo_act(act, (double)x[e]);
+        put_code(packed, e, bits, bucketize(s, nb, x[e]));
+    }
+}
+
+void fbo_fwd_bf16(int act, int bits, const float *s, const uint16_t *x, uint16_t *y,
+                  uint32_t *packed, size_t n)
+{
+    int nb = (1 << bits) - 1;
+    memset(packed, 0, 4 * fbo_packed_words(n, bits));
+    for (size_t e = 0; e < n; ++e) {
+        y[e] = fbo_f64_to_bf16(fbo_act(act, fbo_bf16_to_f64(x[e])));
+        put_code(packed, e, bits, bucketize(s, nb, bf16_to_f32(x[e])));
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Backward, Listing 1: grad_in = grad_out * y[X_pos].  The product is one   */
+/* binary32 multiply (levels are binary32), then one rounding to the dtype.  */
+/* ------------------------------------------------------------------------ */
+void fbo_bwd_f32(int bits, const float *lev, const uint32_t *packed, const float *grad_out,
+                 float *grad_in, size_t n)
+{
+    for (size_t e = 0; e < n; ++e) {
+        volatile float p = grad_out[e] * lev[get_code(packed, e, bits)];
+        grad_in[e] = p;
+    }
+}
+
+void fbo_bwd_bf16(int bits, const float *lev, const uint32_t *packed, const uint16_t *grad_out,
+                  uint16_t *grad_in, size_t n)
+{
+    for (size_t e = 0; e < n; ++e) {
+        volatile float p = bf16_to_f32(grad_out[e]) * lev[get_code(packed, e, bits)];
+        grad_in[e] = fbo_f64_to_bf16((double)p);
+    }
+}
+
+/* Elementwise helpers for the Python side. */
+void fbo_act_array(int act, const double *x, double *y, size_t n)
+{
+    for (size_t e = 0; e < n; ++e) y[e] = fbo_act(act, x[e]);
+}
+
+void fbo_act_deriv_array(int act, const double *x, double *y, size_t n)
+{
+    for (size_t e = 0; e < n; ++e) y[e] = fbo_act_deriv(act, x[e]);
+}
+
+void fbo_f64_to_bf16_array(const double *x, uint16_t *y, size_t n)
+{
+    for (size_t e = 0; e < n; ++e) y[e] = fbo_f64_to_bf16(x[e]);
+}
