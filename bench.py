@@ -1,0 +1,461 @@
+#!/usr/bin/env python
+"""Benchmark of the Few-Bit Backward hot path on B200.
+
+One "step" is one pass of the whole hot path over one batch of the headline
+workload: for every bit width of the workload, the fused forward kernel
+(activation + bucketize + pack) followed by the backward kernel (unpack +
+level lookup + multiply).  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c3|c2|c4|c1]
+
+N > 1 is launched by torchrun; every rank processes its own tensor of the
+workload's shape (the path is elementwise: independent shards, no collective
+on the data path), time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2202_00441_b200 import workloads as wl  # noqa: E402
+
+METRIC = "fused fwd+pack / unpack+bwd elements/s and HBM GB/s vs ~8 TB/s peak"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------
+# helpers
+# ----------------------------------------------------------------------------
+def elem_size(case: wl.Case) -> int:
+    return 4 if case.dtype == "f32" else 2
+
+
+def algorithmic_bytes(case: wl.Case, n: int, bits: int) -> float:
+    """Per kernel launch (forward: x in, y out, codes out; backward: codes in,
+    grad_out in, grad_in out): n * (2 * sizeof(T) + bits / 8)."""
+    return n * (2 * elem_size(case) + bits / 8.0)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        clocks, reasons, mx = [], set(), None
+        try:
+            for line in open(self.path):
+                f = [c.strip() for c in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    clocks.append(float(f[1])); mx = float(f[2])
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if clocks:
+            out.update(sm_mhz=statistics.median(clocks), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(clocks))
+        return out
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, world, local
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ----------------------------------------------------------------------------
+# the CPU oracle as a timed baseline (only this function touches oracle/)
+# ----------------------------------------------------------------------------
+def oracle_pass(case: wl.Case, act: str, x_np, g_np, tables, threads: int) -> float:
+    """One pass of the hot path (all bit widths, forward + backward) through the
+    oracle as it stands, the sample cut into `threads` shards on 32-element
+    boundaries, one oracle call per shard.  Returns seconds."""
+    import concurrent.futures
+
+    import oracle
+
+    n = x_np.size
+    cuts = [wl.shard_range(n, r, threads, 1024) for r in range(threads)]
+
+    def work(rng):
+        lo, hi = rng
+        for bits in case.bits:
+            s, lev = tables[bits]
+            _, p = oracle.fwd(act, bits, s, x_np[lo:hi])
+            oracle.bwd(bits, lev, p, g_np[lo:hi])
+
+    t0 = time.perf_counter()
+    with concurrent.futures.ThreadPoolExecutor(max_workers=threads) as pool:
+        list(pool.map(work, cuts))
+    return time.perf_counter() - t0
+
+
+def oracle_tables(case: wl.Case, act: str):
+    import oracle
+    import numpy as np
+
+    out = {}
+    for bits in case.bits:
+        r = oracle.dp_solve(act, bits)
+        out[bits] = (r["s"].astype(np.float32), r["lev"].astype(np.float32))
+    return out
+
+
+def cpu_baseline(case: wl.Case, act: str, sample_elems: int):
+    import oracle  # noqa: F401  (builds the shared object outside the timed region)
+    threads = len(os.sched_getaffinity(0))
+    x, g = wl.draw(case, "cpu", n=sample_elems)
+    x_np, g_np = wl.to_numpy_bits(x), wl.to_numpy_bits(g)
+    tables = oracle_tables(case, act)
+    secs = oracle_pass(case, act, x_np, g_np, tables, threads)
+    passes = 2 * len(case.bits) * sample_elems
+    return {"value": passes / secs, "unit": "elements/s", "cores": threads, "kind": "oracle",
+            "sample": f"first {sample_elems} elements of the {case.name} draw, bits {list(case.bits)}, fwd+bwd, "
+                      f"{threads} shards on {threads} threads, {secs:.2f} s"}
+
+
+# ----------------------------------------------------------------------------
+# reference arm: the oracle on host cores
+# ----------------------------------------------------------------------------
+def run_reference(args, case: wl.Case, act: str):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle  # noqa: F401
+    threads = len(os.sched_getaffinity(0))
+    sample = args.ref_sample
+    x, g = wl.draw(case, "cpu", n=sample)
+    x_np, g_np = wl.to_numpy_bits(x), wl.to_numpy_bits(g)
+    tables = oracle_tables(case, act)
+    for _ in range(args.warmup):
+        oracle_pass(case, act, x_np, g_np, tables, threads)
+    t = 0.0
+    for _ in range(args.steps):
+        t += oracle_pass(case, act, x_np, g_np, tables, threads)
+    passes = 2 * len(case.bits) * sample * args.steps
+    value = passes / t
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "elements/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": case.dtype, "data": "synthetic",
+        "config": {"workload": case.name, "act": act, "bits": list(case.bits), "elements_per_step_sample": sample,
+                   "note": "CPU oracle on a bounded sample of the workload; elements counted once per kernel-equivalent pass"},
+        "cpu_baseline": {"value": value, "unit": "elements/s", "cores": threads, "kind": "oracle",
+                         "sample": f"first {sample} elements of the {case.name} draw per step"},
+        "e2e": {"value": value, "unit": "elements/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------
+def run_ours(args, case: wl.Case, act: str):
+    import paper_2202_00441_b200 as fb
+
+    rank, world, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    fb.load_library()
+
+    n = case.n
+    x, g = wl.draw(dataclass_replace_seed(case, case.seed + rank), dev)
+    y, gi = torch.empty_like(x), torch.empty_like(g)
+    tables = {b: fb.fewbit_table_create(act, b) for b in case.bits}
+    packed = {b: torch.empty(fb.fewbit_packed_bytes(n, b) // 4, dtype=torch.int32, device=dev) for b in case.bits}
+    footprint = (x.numel() * x.element_size()) * 4 + sum(p.numel() * 4 for p in packed.values())
+    flush = None
+    if footprint < 512 * 2 ** 20:            # smaller than a few L2s: flush between launches
+        flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+
+    launches = [("fwd", b) for b in case.bits] + [("bwd", b) for b in case.bits]
+    order = [(kind, b) for b in case.bits for kind in ("fwd", "bwd")]
+
+    def one_step(events=None):
+        for i, (kind, b) in enumerate(order):
+            if flush is not None:
+                flush.zero_()
+            if events is not None:
+                events[i][0].record()
+            if kind == "fwd":
+                fb.fewbit_fwd(tables[b], x, y, packed[b])
+            else:
+                fb.fewbit_bwd(tables[b], packed[b], g, gi)
+            if events is not None:
+                events[i][1].record()
+
+    for _ in range(args.warmup):
+        one_step()
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in order]
+          for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    barrier(world)
+    launches_before = fb.fewbit_launch_count()
+    start.record()
+    for s in range(args.steps):
+        one_step(ev[s])
+    stop.record()
+    barrier(world)
+    launches_in_region = fb.fewbit_launch_count() - launches_before
+    clocks = sampler.stop() if rank == 0 else None
+    if flush is None:
+        total_ms = start.elapsed_time(stop)
+    else:                                      # the flush writes are not part of the path: sum the launches
+        total_ms = sum(a.elapsed_time(b) for step in ev for a, b in step)
+    total_ms = max_over_ranks(total_ms, world, dev)
+
+    per_kernel = {}
+    for i, (kind, b) in enumerate(order):
+        ms = [ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(args.steps)]
+        avg = sum(ms) / len(ms)
+        by = algorithmic_bytes(case, n, b)
+        per_kernel[f"{kind}_k{b}"] = {"avg_us": 1e3 * avg, "min_us": 1e3 * min(ms), "gbs": by / (avg * 1e-3) / 1e9,
+                                      "gelems": n / (avg * 1e-3) / 1e9, "bytes": by}
+    peak, peak_kind = measured_peak()
+    dom = max(per_kernel, key=lambda k: per_kernel[k]["avg_us"])
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": per_kernel[dom]["gbs"], "peak": peak, "unit": "GB/s",
+                "frac": per_kernel[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}",
+                "frac_of_nominal_8TBs": per_kernel[dom]["gbs"] / NOMINAL_HBM_GBS,
+                "traffic": NCU_TRAFFIC_BYTES_PER_ELEM.get((case.dtype, dom)) and
+                NCU_TRAFFIC_BYTES_PER_ELEM[(case.dtype, dom)] * n}
+    elems_per_step = 2 * len(case.bits) * n
+    value = world * elems_per_step * args.steps / (total_ms * 1e-3)
+    bytes_per_step = 2 * sum(algorithmic_bytes(case, n, b) for b in case.bits)
+
+    # ---- end to end through the host-buffer entry points -----------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        hx, hg = x.cpu().pin_memory(), g.cpu().pin_memory()
+        hy, hgi = torch.empty_like(hx).pin_memory(), torch.empty_like(hg).pin_memory()
+        hp = {b: torch.empty(packed[b].numel(), dtype=torch.int32).pin_memory() for b in case.bits}
+        ws = torch.empty(fb.fewbit_host_workspace_bytes(1 << 23, x.dtype, max(case.bits)), dtype=torch.uint8, device=dev)
+
+        def e2e_step():
+            for b in case.bits:
+                fb.fewbit_fwd_host(tables[b], hx, hy, hp[b], ws)
+                fb.fewbit_bwd_host(tables[b], hp[b], hg, hgi, ws)
+
+        e2e_step()
+        barrier(world)
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        barrier(world)
+        secs = max_over_ranks(time.perf_counter() - t0, world, dev)
+        eb = elem_size(case)
+        h2d = sum(n * eb + (n * eb + packed[b].numel() * 4) for b in case.bits)
+        d2h = sum((n * eb + packed[b].numel() * 4) + n * eb for b in case.bits)
+        e2e = {"value": world * elems_per_step * args.e2e_steps / secs, "unit": "elements/s",
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
+               "gbs_pcie_each_way": h2d * args.e2e_steps / secs / 1e9,
+               "api": "fewbit_fwd_host / fewbit_bwd_host on pinned host tensors"}
+        del hx, hg, hy, hgi, hp, ws
+
+    # ---- plain unfused PyTorch activation (context) -----------------------------------------------
+    torch_ref = None
+    if rank == 0 and not args.no_torch_baseline:
+        torch_ref = torch_unfused(case, act, x, g)
+
+    # ---- the other configurations, quick device-resident runs (context) --------------------------
+    also = {}
+    if rank == 0 and not args.no_also:
+        for name in ("c2", "c4", "c1"):
+            if wl.CONFIGS[name].name != case.name:
+                also[name] = quick_config(fb, wl.CONFIGS[name], dev)
+
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(case, act, args.cpu_sample)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "elements/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": case.dtype, "data": "synthetic",
+            "config": {"workload": case.name, "act": act, "bits": list(case.bits), "shape": list(case.shape),
+                       "elements": n, "launches_per_step": len(order),
+                       "l2": "inputs larger than L2 (no flush)" if flush is None else "256 MiB flush write before every launch; value sums the launches",
+                       "elements_counted": "once per kernel pass (forward and backward each count n)",
+                       "parallelism": f"independent shards x{world}"},
+            "hbm_gbs": world * bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9,
+            "hbm_frac_of_nominal_8TBs": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            "hbm_frac_of_measured_copy": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9 / peak,
+            "roofline": roofline, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": launches_in_region, "clocks": clocks, "torch_unfused": torch_ref, "also": also,
+            "saved_activation_ratio": {str(b): 8 * elem_size(case) / b for b in case.bits},
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum of one launch / n) read from the
+# ncu captures summarised under profiles/; None until a capture exists for that kernel.
+NCU_TRAFFIC_BYTES_PER_ELEM = {}
+
+
+def dataclass_replace_seed(case: wl.Case, seed: int) -> wl.Case:
+    import dataclasses
+    return dataclasses.replace(case, seed=seed)
+
+
+def torch_unfused(case: wl.Case, act: str, x, g, reps: int = 5):
+    import torch.nn.functional as F
+    fn = {"gelu": F.gelu, "silu": F.silu, "sigmoid": torch.sigmoid, "tanh": torch.tanh, "elu": F.elu,
+          "softplus": F.softplus, "leaky_relu": F.leaky_relu}[act]
+    xr = x.detach().clone().requires_grad_(True)
+    a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    fwd_ms, bwd_ms = [], []
+    for i in range(reps + 2):
+        a.record()
+        out = fn(xr)
+        b.record()
+        out.backward(g)
+        c.record()
+        torch.cuda.synchronize()
+        xr.grad = None
+        if i >= 2:
+            fwd_ms.append(a.elapsed_time(b)); bwd_ms.append(b.elapsed_time(c))
+        del out
+    n, eb = case.n, elem_size(case)
+    return {"fwd_us": 1e3 * min(fwd_ms), "bwd_us": 1e3 * min(bwd_ms),
+            "fwd_gbs": 2 * eb * n / (min(fwd_ms) * 1e-3) / 1e9, "bwd_gbs": 3 * eb * n / (min(bwd_ms) * 1e-3) / 1e9,
+            "saved_bytes_per_elem": eb, "note": "stock torch forward + autograd backward, full input kept"}
+
+
+def quick_config(fb, case: wl.Case, dev, reps: int = 10):
+    """Device-resident timing of another configuration, L2 flushed before every launch."""
+    x, g = wl.draw(case, dev)
+    y, gi = torch.empty_like(x), torch.empty_like(g)
+    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+    out = {}
+    for act in case.acts:
+        for b in case.bits:
+            t = fb.fewbit_table_create(act, b)
+            p = torch.empty(fb.fewbit_packed_bytes(case.n, b) // 4, dtype=torch.int32, device=dev)
+            f_ms, b_ms = [], []
+            for i in range(reps + 3):
+                e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+                flush.zero_(); e[0].record(); fb.fewbit_fwd(t, x, y, p); e[1].record()
+                flush.zero_(); e[2].record(); fb.fewbit_bwd(t, p, g, gi); e[3].record()
+                torch.cuda.synchronize()
+                if i >= 3:
+                    f_ms.append(e[0].elapsed_time(e[1])); b_ms.append(e[2].elapsed_time(e[3]))
+            by = algorithmic_bytes(case, case.n, b)
+            fm, bm = statistics.median(f_ms), statistics.median(b_ms)
+            out[f"{act}_k{b}"] = {"fwd_us": 1e3 * fm, "bwd_us": 1e3 * bm, "fwd_gbs": by / (fm * 1e-3) / 1e9,
+                                  "bwd_gbs": by / (bm * 1e-3) / 1e9}
+    return {"workload": case.name, "elements": case.n, "dtype": case.dtype, "l2": "flushed before every launch",
+            "cases": out}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=sorted(wl.CONFIGS), default="c3")
+    ap.add_argument("--act", default=None, help="activation of the workload to time (default: its first)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-sample", type=int, default=1 << 23)
+    ap.add_argument("--ref-sample", type=int, default=1 << 22)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-torch-baseline", action="store_true")
+    ap.add_argument("--no-also", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    case = wl.CONFIGS[args.workload]
+    act = args.act or case.acts[0]
+    if args.impl == "reference":
+        run_reference(args, case, act)
+    else:
+        run_ours(args, case, act)
+
+
+if __name__ == "__main__":
+    main()

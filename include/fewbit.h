@@ -1,0 +1,202 @@
+/*
+ * fewbit.h -- C ABI of the Few-Bit Backward hot path for NVIDIA B200 (sm_100a).
+ *
+ * The method (arXiv 2202.00441): a pointwise activation f keeps, for its
+ * backward pass, not the input x but only the index of the interval of a
+ * piecewise-constant approximation q of f' that x falls into (Eq. 2), i.e.
+ * `bits` = log2(K) bits per element.  Backward multiplies grad_out by the
+ * level of that interval instead of f'(x) (Listing 1).  The intervals and
+ * levels minimise the L2 error of Eq. 3 and are found once, offline, by the
+ * dynamic programme of Eq. 7-9.
+ *
+ * Conventions that hold for every call
+ *   - plain C types only; every pointer is commented HOST or DEVICE;
+ *   - the library never throws, never calls exit(), never synchronises the
+ *     device in the DEVICE-pointer calls and never allocates device memory;
+ *     the only allocation is the host-side table object;
+ *   - the caller owns every buffer; a table is immutable after creation and
+ *     may be used from many threads and streams at once;
+ *   - every function that can fail returns a fewbit_status.
+ *
+ * Table layout: K = 2^bits levels lev[0..K-1] and K-1 interior boundaries
+ * s[0..K-2] (non-decreasing), both binary32.  The code of x is
+ *     code(x) = #{ j : s[j] < x }        (strict, compared in binary32)
+ * so interval i is (s[i-1], s[i]], anything below s[0] has code 0, anything
+ * above s[K-2] has code K-1, and NaN has code 0.
+ *
+ * Saved-tensor layout ("packed"): one flat bit stream, element e occupies
+ * bits [e*bits, e*bits + bits), least significant bit first, stored in
+ * little-endian 32-bit words.  32 consecutive elements always fill exactly
+ * `bits` words.  Unused high bits of the last word are written as zero.
+ */
+#ifndef FEWBIT_H_
+#define FEWBIT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define FEWBIT_API
+#else
+#define FEWBIT_API __attribute__((visibility("default")))
+#endif
+
+typedef struct fewbit_table fewbit_table;
+
+/* Activations f (Sec. 2; the rows of Table 1 plus ELU and LeakyReLU). */
+typedef enum fewbit_act {
+    FEWBIT_GELU = 0,       /* x * Phi(x), the erf form                       */
+    FEWBIT_SILU = 1,       /* x * sigmoid(x)  (Swish)                        */
+    FEWBIT_SIGMOID = 2,    /* 1 / (1 + exp(-x))                              */
+    FEWBIT_TANH = 3,
+    FEWBIT_ELU = 4,        /* x > 0 ? x : exp(x) - 1        (alpha = 1)      */
+    FEWBIT_SOFTPLUS = 5,   /* log(1 + exp(x))               (beta = 1)       */
+    FEWBIT_LEAKY_RELU = 6  /* x > 0 ? x : 0.01 x                             */
+} fewbit_act;
+#define FEWBIT_NUM_ACTS 7
+
+typedef enum fewbit_dtype {
+    FEWBIT_F32 = 0,        /* IEEE binary32                                  */
+    FEWBIT_BF16 = 1        /* bfloat16                                       */
+} fewbit_dtype;
+
+typedef enum fewbit_status {
+    FEWBIT_OK = 0,
+    FEWBIT_ERR_INVALID_ARG = 1,   /* NULL pointer, bits outside 1..4, bad enum, unsorted table */
+    FEWBIT_ERR_UNSUPPORTED = 2,   /* valid request this build cannot serve                      */
+    FEWBIT_ERR_ALIGNMENT = 3,     /* a buffer breaks the alignment rule of the call             */
+    FEWBIT_ERR_CUDA = 4,          /* a CUDA call failed; see fewbit_last_cuda_error()           */
+    FEWBIT_ERR_ALLOC = 5          /* host allocation failed / workspace too small               */
+} fewbit_status;
+
+/* ------------------------------------------------------------------------- */
+/* Tables (Eq. 2: parameters s and y; solved by Eq. 7-9, levels by Eq. 4)     */
+/* ------------------------------------------------------------------------- */
+
+/*
+ * Optimal `bits`-bit table for `act`: the dynamic programme of Eq. 7 over a
+ * uniform grid of 4096 cells on [-8, 8] with the uniform weight of Eq. 10
+ * (A = -8, B = 8), prefix integrals as in Eq. 8-9, levels by Eq. 4.  Runs on
+ * the CPU (a fraction of a second; results are cached per activation).
+ * Returns a HOST handle, or NULL when act/bits are invalid or memory is
+ * exhausted.  Release with fewbit_table_destroy().
+ */
+FEWBIT_API fewbit_table *fewbit_table_create(fewbit_act act, int bits);
+
+/*
+ * Same solver with explicit range [A, B] and number of grid cells
+ * (2^bits <= n_cells <= 65536).  *out (HOST) receives the handle.
+ */
+FEWBIT_API fewbit_status fewbit_table_create_ex(fewbit_act act, int bits, double A, double B,
+                                                int n_cells, fewbit_table **out);
+
+/*
+ * Table from caller-supplied parameters (Listing 1's globally stored s, y):
+ * s = 2^bits - 1 boundaries, lev = 2^bits levels, both HOST binary32 arrays,
+ * copied.  s must be non-decreasing and free of NaN, else
+ * FEWBIT_ERR_INVALID_ARG.
+ */
+FEWBIT_API fewbit_status fewbit_table_from_arrays(fewbit_act act, int bits, const float *s,
+                                                  const float *lev, fewbit_table **out);
+
+/* Frees a table; NULL is accepted. */
+FEWBIT_API void fewbit_table_destroy(fewbit_table *table);
+
+/*
+ * Reads a table back.  Any output pointer (all HOST) may be NULL.
+ * s_out needs room for 2^bits - 1 floats, lev_out for 2^bits floats.
+ * *objective is the value of Eq. 3 reached by the solver (NaN for a table
+ * made by fewbit_table_from_arrays).
+ */
+FEWBIT_API fewbit_status fewbit_table_get(const fewbit_table *table, int *act, int *bits,
+                                          float *s_out, float *lev_out, double *objective);
+
+/* Bytes of the saved tensor for n elements: 4 * ceil(n * bits / 32); 0 if bits is invalid. */
+FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
+
+/* ------------------------------------------------------------------------- */
+/* Hot path on DEVICE buffers (Listing 1)                                     */
+/* ------------------------------------------------------------------------- */
+
+/*
+ * Forward half, one kernel launch on `stream` (a cudaStream_t passed as
+ * void*; NULL = the legacy default stream), asynchronous:
+ *     y[e]      = f(x[e])                 exact activation, rounded to dtype
+ *     code[e]   = #{ j : s[j] < x[e] }    Eq. 2 / "sortedsearch" of Listing 1
+ *     packed    = the codes as a `bits`-bit stream (layout above)
+ * x, y: DEVICE, n elements of `dtype`, 32-byte aligned; y == x (exact alias)
+ * is allowed, any other overlap is undefined.  packed: DEVICE,
+ * fewbit_packed_bytes(n, bits) bytes, 16-byte aligned; nothing beyond those
+ * bytes is written.  n == 0 returns FEWBIT_OK without a launch.
+ * Errors: FEWBIT_ERR_INVALID_ARG (NULL table or buffer, bad dtype),
+ * FEWBIT_ERR_ALIGNMENT, FEWBIT_ERR_CUDA (launch failed).
+ */
+FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y,
+                                    uint32_t *packed, size_t n, fewbit_dtype dtype, void *stream);
+
+/*
+ * Backward half, one kernel launch on `stream`, asynchronous:
+ *     grad_in[e] = round_dtype( (float)grad_out[e] * lev[code[e]] )
+ * (Eq. 1 with f' replaced by q of Eq. 2; one binary32 multiply, one rounding).
+ * packed: DEVICE, as written by fewbit_fwd with a table of the same `bits`,
+ * 16-byte aligned.  grad_out, grad_in: DEVICE, n elements of `dtype`,
+ * 32-byte aligned; grad_in == grad_out allowed.  Errors as fewbit_fwd.
+ */
+FEWBIT_API fewbit_status fewbit_bwd(const fewbit_table *table, const uint32_t *packed,
+                                    const void *grad_out, void *grad_in, size_t n,
+                                    fewbit_dtype dtype, void *stream);
+
+/* ------------------------------------------------------------------------- */
+/* Hot path on HOST buffers                                                   */
+/* ------------------------------------------------------------------------- */
+
+/*
+ * Device bytes fewbit_fwd_host / fewbit_bwd_host need in `workspace` to
+ * stream `chunk_elems` elements per pipeline stage (rounded up to a multiple
+ * of 1024 elements; the pipeline has 3 stages).
+ */
+FEWBIT_API size_t fewbit_host_workspace_bytes(size_t chunk_elems, fewbit_dtype dtype, int bits);
+
+/*
+ * Forward half on HOST buffers: x_host -> (y_host, packed_host), same
+ * results as fewbit_fwd.  The tensor is cut into chunks; each chunk is copied
+ * to `workspace` (DEVICE, caller-owned, 256-byte aligned, `workspace_bytes`
+ * long), run through the forward kernel and copied back, with the copies of
+ * neighbouring chunks overlapping the kernel on three internal streams.
+ * Blocks until the results are in host memory.  Page-locked host buffers are
+ * needed for the copies to overlap; pageable ones work, slower.
+ * FEWBIT_ERR_ALLOC if the workspace cannot hold one 1024-element chunk.
+ * Calls on the same device that overlap in time must use disjoint workspaces.
+ */
+FEWBIT_API fewbit_status fewbit_fwd_host(const fewbit_table *table, const void *x_host,
+                                         void *y_host, uint32_t *packed_host, size_t n,
+                                         fewbit_dtype dtype, void *workspace,
+                                         size_t workspace_bytes);
+
+/* Backward half on HOST buffers: (packed_host, grad_out_host) -> grad_in_host; see fewbit_fwd_host. */
+FEWBIT_API fewbit_status fewbit_bwd_host(const fewbit_table *table, const uint32_t *packed_host,
+                                         const void *grad_out_host, void *grad_in_host, size_t n,
+                                         fewbit_dtype dtype, void *workspace,
+                                         size_t workspace_bytes);
+
+/* ------------------------------------------------------------------------- */
+/* Diagnostics                                                                */
+/* ------------------------------------------------------------------------- */
+
+/* Static, never NULL. */
+FEWBIT_API const char *fewbit_status_string(fewbit_status status);
+
+/* The cudaError_t (as int) behind the calling thread's last FEWBIT_ERR_CUDA; 0 if none. */
+FEWBIT_API int fewbit_last_cuda_error(void);
+
+/* Kernels launched by this library in this process so far (all threads). */
+FEWBIT_API uint64_t fewbit_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FEWBIT_H_ */

@@ -1,0 +1,252 @@
+// Host side of the library: the table object and the offline solver that
+// finds the optimal piecewise-constant approximation of f' (Eq. 3) by the
+// dynamic programme of Eq. 7 over prefix integrals (Eq. 8-9), with the
+// levels of Eq. 4.  Pure C++17, no CUDA.
+#include "fewbit_internal.h"
+
+#include <cmath>
+#include <cstring>
+#include <limits>
+#include <map>
+#include <memory>
+#include <mutex>
+#include <new>
+#include <tuple>
+#include <vector>
+
+namespace fewbit {
+namespace {
+
+// ---------------------------------------------------------------------------
+// f and f' in binary64 (Sec. 2; Eq. 1 needs f', the closed form of Eq. 9's
+// FW needs f).
+// ---------------------------------------------------------------------------
+inline double logistic(double x) {
+    if (x >= 0.0) return 1.0 / (1.0 + std::exp(-x));
+    const double e = std::exp(x);
+    return e / (1.0 + e);
+}
+
+inline double Phi(double x) { return 0.5 * std::erfc(-x * 0.70710678118654752440); }
+inline double phi(double x) { return 0.39894228040143267794 * std::exp(-0.5 * x * x); }
+
+double value(fewbit_act a, double x) {
+    switch (a) {
+    case FEWBIT_GELU: return x * Phi(x);
+    case FEWBIT_SILU: return x * logistic(x);
+    case FEWBIT_SIGMOID: return logistic(x);
+    case FEWBIT_TANH: return std::tanh(x);
+    case FEWBIT_ELU: return x > 0.0 ? x : std::expm1(x);
+    case FEWBIT_SOFTPLUS: return std::fmax(x, 0.0) + std::log1p(std::exp(-std::fabs(x)));
+    case FEWBIT_LEAKY_RELU: return x > 0.0 ? x : 0.01 * x;
+    }
+    return std::numeric_limits<double>::quiet_NaN();
+}
+
+double slope(fewbit_act a, double x) {
+    switch (a) {
+    case FEWBIT_GELU: return Phi(x) + x * phi(x);
+    case FEWBIT_SILU: { const double g = logistic(x); return g + x * g * (1.0 - g); }
+    case FEWBIT_SIGMOID: { const double g = logistic(x); return g * (1.0 - g); }
+    case FEWBIT_TANH: { const double t = std::tanh(x); return (1.0 - t) * (1.0 + t); }
+    case FEWBIT_ELU: return x > 0.0 ? 1.0 : std::exp(x);
+    case FEWBIT_SOFTPLUS: return logistic(x);
+    case FEWBIT_LEAKY_RELU: return x > 0.0 ? 1.0 : 0.01;
+    }
+    return std::numeric_limits<double>::quiet_NaN();
+}
+
+// ---------------------------------------------------------------------------
+// One solved grid: every layer DP(., k), k = 1..kMaxLevels, with its argmin,
+// so that tables for 1, 2, 3 and 4 bits come out of a single run.
+// ---------------------------------------------------------------------------
+struct Solved {
+    int n = 0;
+    double A = 0, B = 0;
+    std::vector<double> F2, FW, Wt;             // prefix integrals of Eq. 8-9 (uniform weight, Eq. 10)
+    std::vector<double> best_at_n;              // DP(n, k)
+    std::vector<std::vector<int32_t>> from;     // from[k][i] = argmin_j of Eq. 7
+
+    double level(int j, int i) const { return (FW[i] - FW[j]) / (Wt[i] - Wt[j]); }
+};
+
+std::shared_ptr<const Solved> solve_grid(fewbit_act act, double A, double B, int n) {
+    auto out = std::make_shared<Solved>();
+    Solved &g = *out;
+    g.n = n; g.A = A; g.B = B;
+    g.F2.assign(n + 1, 0.0); g.FW.assign(n + 1, 0.0); g.Wt.assign(n + 1, 0.0);
+
+    // Eq. 9: the three running integrals.  With w = 1 on [A,B] the integral of
+    // f' is f itself; the integral of f'^2 uses a 4-node Gauss-Legendre rule
+    // per cell, whose nodes never touch a grid point (f' may jump there).
+    const double node[2] = {0.33998104358485626480, 0.86113631159405257522};
+    const double wght[2] = {0.65214515486254614263, 0.34785484513745385737};
+    const double fA = value(act, A);
+    double left = A;
+    for (int i = 1; i <= n; ++i) {
+        const double right = (i == n) ? B : A + (B - A) * (static_cast<double>(i) / n);
+        const double c = 0.5 * (left + right), r = 0.5 * (right - left);
+        double q = 0.0;
+        for (int m = 0; m < 2; ++m) {
+            const double dm = slope(act, c - r * node[m]), dp = slope(act, c + r * node[m]);
+            q += wght[m] * (dm * dm + dp * dp);
+        }
+        g.F2[i] = g.F2[i - 1] + r * q;
+        g.FW[i] = value(act, right) - fA;
+        g.Wt[i] = right - A;
+        left = right;
+    }
+
+    // Eq. 7 with Eq. 8's O(1) cost: cost(j,i) = dF2 - dFW^2 / dW, never below 0.
+    const double inf = std::numeric_limits<double>::infinity();
+    std::vector<double> prev(n + 1, inf), cur(n + 1, inf);
+    prev[0] = 0.0;                                  // zero pieces cover [A, A]
+    g.best_at_n.assign(kMaxLevels + 1, inf);
+    g.from.assign(kMaxLevels + 1, {});
+    const int layers = std::min(kMaxLevels, n);
+    for (int k = 1; k <= layers; ++k) {
+        std::vector<int32_t> &arg = g.from[k];
+        arg.assign(n + 1, -1);
+        std::fill(cur.begin(), cur.end(), inf);
+        for (int i = k; i <= n; ++i) {
+            const double f2i = g.F2[i], fwi = g.FW[i], wi = g.Wt[i];
+            double best = inf;
+            int32_t best_j = -1;
+            for (int j = k - 1; j < i; ++j) {
+                const double dfw = fwi - g.FW[j];
+                double cost = (f2i - g.F2[j]) - dfw * (dfw / (wi - g.Wt[j]));
+                cost = cost > 0.0 ? cost : 0.0;
+                const double total = prev[j] + cost;
+                if (total < best) { best = total; best_j = j; }
+            }
+            cur[i] = best;
+            arg[i] = best_j;
+        }
+        g.best_at_n[k] = cur[n];
+        prev.swap(cur);
+    }
+    return out;
+}
+
+std::mutex g_cache_mutex;
+std::map<std::tuple<int, double, double, int>, std::shared_ptr<const Solved>> g_cache;
+
+std::shared_ptr<const Solved> solved_for(fewbit_act act, double A, double B, int n) {
+    const auto key = std::make_tuple(static_cast<int>(act), A, B, n);
+    {
+        std::lock_guard<std::mutex> lock(g_cache_mutex);
+        auto it = g_cache.find(key);
+        if (it != g_cache.end()) return it->second;
+    }
+    auto fresh = solve_grid(act, A, B, n);
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    if (g_cache.size() >= 64) g_cache.clear();
+    return g_cache.emplace(key, fresh).first->second;
+}
+
+bool valid_act(int a) { return a >= 0 && a < FEWBIT_NUM_ACTS; }
+bool valid_bits(int b) { return b >= 1 && b <= 4; }
+
+}  // namespace
+}  // namespace fewbit
+
+using fewbit::kMaxLevels;
+
+extern "C" {
+
+fewbit_status fewbit_table_create_ex(fewbit_act act, int bits, double A, double B, int n_cells,
+                                     fewbit_table **out) {
+    if (out == nullptr) return FEWBIT_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!fewbit::valid_act(act) || !fewbit::valid_bits(bits)) return FEWBIT_ERR_INVALID_ARG;
+    const int K = 1 << bits;
+    if (!(A < B) || !std::isfinite(A) || !std::isfinite(B) || n_cells < K || n_cells > 65536)
+        return FEWBIT_ERR_INVALID_ARG;
+    try {
+        auto g = fewbit::solved_for(act, A, B, n_cells);
+        // walk the argmins back from (n, K): right ends of pieces K, K-1, ..., 1
+        int ends[kMaxLevels + 1];
+        ends[K] = g->n;
+        for (int k = K; k >= 1; --k) ends[k - 1] = g->from[k][ends[k]];
+        auto *t = new fewbit_table();
+        t->act = act;
+        t->bits = bits;
+        t->objective = g->best_at_n[K];
+        for (int m = 0; m < kMaxLevels; ++m) { t->s[m] = std::numeric_limits<float>::infinity(); t->lev[m] = 0.0f; }
+        for (int m = 1; m < K; ++m) {
+            const int i = ends[m];
+            const double sm = (i == g->n) ? B : A + (B - A) * (static_cast<double>(i) / g->n);
+            t->s[m - 1] = static_cast<float>(sm);
+        }
+        for (int m = 0; m < K; ++m) t->lev[m] = static_cast<float>(g->level(ends[m], ends[m + 1]));   // Eq. 4
+        *out = t;
+        return FEWBIT_OK;
+    } catch (const std::bad_alloc &) {
+        return FEWBIT_ERR_ALLOC;
+    } catch (...) {
+        return FEWBIT_ERR_UNSUPPORTED;
+    }
+}
+
+fewbit_table *fewbit_table_create(fewbit_act act, int bits) {
+    fewbit_table *t = nullptr;
+    if (fewbit_table_create_ex(act, bits, -8.0, 8.0, 4096, &t) != FEWBIT_OK) return nullptr;
+    return t;
+}
+
+fewbit_status fewbit_table_from_arrays(fewbit_act act, int bits, const float *s, const float *lev,
+                                       fewbit_table **out) {
+    if (out == nullptr) return FEWBIT_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!fewbit::valid_act(act) || !fewbit::valid_bits(bits) || s == nullptr || lev == nullptr)
+        return FEWBIT_ERR_INVALID_ARG;
+    const int K = 1 << bits;
+    for (int m = 0; m < K - 1; ++m) {
+        if (std::isnan(s[m])) return FEWBIT_ERR_INVALID_ARG;
+        if (m > 0 && s[m] < s[m - 1]) return FEWBIT_ERR_INVALID_ARG;
+    }
+    auto *t = new (std::nothrow) fewbit_table();
+    if (t == nullptr) return FEWBIT_ERR_ALLOC;
+    t->act = act;
+    t->bits = bits;
+    t->objective = std::numeric_limits<double>::quiet_NaN();
+    for (int m = 0; m < kMaxLevels; ++m) { t->s[m] = std::numeric_limits<float>::infinity(); t->lev[m] = 0.0f; }
+    // +0 and -0 compare equal; store +0 so that every kernel variant sees one pattern
+    for (int m = 0; m < K - 1; ++m) t->s[m] = (s[m] == 0.0f) ? 0.0f : s[m];
+    for (int m = 0; m < K; ++m) t->lev[m] = lev[m];
+    *out = t;
+    return FEWBIT_OK;
+}
+
+void fewbit_table_destroy(fewbit_table *table) { delete table; }
+
+fewbit_status fewbit_table_get(const fewbit_table *table, int *act, int *bits, float *s_out,
+                               float *lev_out, double *objective) {
+    if (table == nullptr) return FEWBIT_ERR_INVALID_ARG;
+    const int K = 1 << table->bits;
+    if (act) *act = static_cast<int>(table->act);
+    if (bits) *bits = table->bits;
+    if (s_out) std::memcpy(s_out, table->s, sizeof(float) * (K - 1));
+    if (lev_out) std::memcpy(lev_out, table->lev, sizeof(float) * K);
+    if (objective) *objective = table->objective;
+    return FEWBIT_OK;
+}
+
+size_t fewbit_packed_bytes(size_t n, int bits) {
+    if (!fewbit::valid_bits(bits)) return 0;
+    return 4 * ((n * static_cast<size_t>(bits) + 31) / 32);
+}
+
+const char *fewbit_status_string(fewbit_status status) {
+    switch (status) {
+    case FEWBIT_OK: return "ok";
+    case FEWBIT_ERR_INVALID_ARG: return "invalid argument";
+    case FEWBIT_ERR_UNSUPPORTED: return "unsupported";
+    case FEWBIT_ERR_ALIGNMENT: return "buffer alignment";
+    case FEWBIT_ERR_CUDA: return "CUDA error";
+    case FEWBIT_ERR_ALLOC: return "allocation failed or workspace too small";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,327 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on
+identical seeded inputs.
+
+Bar: packed words and grad_in bit-identical; y within 2 ulp of the storage
+dtype of the exactly rounded binary64 value.  Both sides use the SAME table
+(read back from the library with fewbit_table_get), so the comparison isolates
+the hot path; the solver is compared with the oracle's DP in the CPU tests.
+"""
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2202_00441_b200 as fb
+from paper_2202_00441_b200 import workloads as wl
+from helpers import bf16_bits_to_f32, finite_mask, ulp_distance
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+GUARD = 64            # guard elements / words placed around every output buffer
+TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16}
+_POOL = ThreadPoolExecutor(max_workers=8)
+_TABLES = {}
+
+
+def table(act, bits):
+    key = (act, bits)
+    if key not in _TABLES:
+        _TABLES[key] = fb.fewbit_table_create(act, bits)
+    return _TABLES[key]
+
+
+def np_bits(t: torch.Tensor) -> np.ndarray:
+    return wl.to_numpy_bits(t)
+
+
+def guarded(n, dtype, fill):
+    """A device buffer of n elements with GUARD canary elements on both sides.
+    The payload starts 256-byte aligned."""
+    pad = 256 // torch.empty(0, dtype=dtype).element_size()
+    assert GUARD <= pad
+    buf = torch.full((n + 2 * pad,), fill, dtype=dtype, device=DEV)
+    return buf, buf[pad:pad + n], pad
+
+
+def check_guards(buf, n, pad, fill):
+    assert bool((buf[:pad] == fill).all()) and bool((buf[pad + n:] == fill).all()), "wrote outside the buffer"
+
+
+def run_gpu(act, bits, x, g, inplace=False):
+    """fwd + bwd through the C ABI with canaries around every output."""
+    t = table(act, bits)
+    n = x.numel()
+    words = fb.fewbit_packed_bytes(n, bits) // 4
+    pbuf, packed, ppad = guarded(words, torch.int32, 0x5A5A5A5A)
+    if inplace:
+        y, gi = x.clone(), g.clone()
+        fb.fewbit_fwd(t, y, y, packed)
+        fb.fewbit_bwd(t, packed, gi, gi)
+    else:
+        fill = 777.0
+        ybuf, y, ypad = guarded(n, x.dtype, fill)
+        gbuf, gi, gpad = guarded(n, x.dtype, fill)
+        fb.fewbit_fwd(t, x, y, packed)
+        fb.fewbit_bwd(t, packed, g, gi)
+        torch.cuda.synchronize()
+        check_guards(ybuf, n, ypad, fill)
+        check_guards(gbuf, n, gpad, fill)
+    torch.cuda.synchronize()
+    check_guards(pbuf, words, ppad, 0x5A5A5A5A)
+    return y, packed, gi
+
+
+def oracle_block(act, bits, s, lev, x_np, g_np):
+    y, p = oracle.fwd(act, bits, s, x_np)
+    gi = oracle.bwd(bits, lev, p, g_np)
+    return y, p, gi
+
+
+def compare_block(act, bits, x_np, g_np, y_np, p_np, gi_np, what):
+    s, lev = table(act, bits).arrays()
+    y_ref, p_ref, gi_ref = oracle_block(act, bits, s, lev, x_np, g_np)
+    assert np.array_equal(p_np[:p_ref.size], p_ref), f"{what}: packed codes differ"
+    assert np.array_equal(gi_np.view(np.uint16 if gi_np.dtype == np.uint16 else np.uint32),
+                          gi_ref.view(np.uint16 if gi_ref.dtype == np.uint16 else np.uint32)), f"{what}: grad_in differs"
+    ok = finite_mask(x_np)
+    d = ulp_distance(y_np[ok], y_ref[ok])
+    assert d.size == 0 or d.max() <= 2, f"{what}: y off by {d.max()} ulp"
+
+
+def compare_full(act, bits, x, g, y, packed, gi, what):
+    compare_block(act, bits, np_bits(x), np_bits(g), np_bits(y), np_bits(packed).view(np.uint32), np_bits(gi), what)
+
+
+def compare_sampled(act, bits, x, g, y, packed, gi, what, blocks=24, block_elems=8192, seed=0):
+    """Element-by-element comparison on randomly placed 32-aligned blocks plus
+    the first and the last (ragged) block."""
+    n = x.numel()
+    rng = np.random.default_rng(seed)
+    starts = {0, max(0, (n - block_elems) // 32 * 32)}
+    while len(starts) < blocks:
+        starts.add(int(rng.integers(0, max(1, n - block_elems))) // 32 * 32)
+    jobs = []
+    for e0 in sorted(starts):
+        m = min(block_elems, n - e0)
+        w0 = e0 // 32 * bits
+        w1 = (((e0 + m) * bits) + 31) // 32
+        jobs.append((e0, np_bits(x[e0:e0 + m]), np_bits(g[e0:e0 + m]), np_bits(y[e0:e0 + m]),
+                     np_bits(packed[w0:w1]).view(np.uint32), np_bits(gi[e0:e0 + m])))
+    list(_POOL.map(lambda j: compare_block(act, bits, j[1], j[2], j[3], j[4], j[5], f"{what} @ {j[0]}"), jobs))
+
+
+# --------------------------------------------------------------------------
+# the five configurations
+# --------------------------------------------------------------------------
+def test_config1_gelu3_f32_full():
+    x, g = wl.draw(wl.C1, DEV)
+    for act in wl.C1.acts:
+        for bits in wl.C1.bits:
+            y, p, gi = run_gpu(act, bits, x, g)
+            compare_full(act, bits, x, g, y, p, gi, "c1")
+
+
+def test_config2_silu_bf16_full():
+    x, g = wl.draw(wl.C2, DEV)
+    for bits in wl.C2.bits:
+        y, p, gi = run_gpu("silu", bits, x, g)
+        n = x.numel()
+        cuts = [wl.shard_range(n, r, 8, 1024) for r in range(8)]
+        jobs = []
+        for lo, hi in cuts:
+            jobs.append(("silu", bits, np_bits(x[lo:hi]), np_bits(g[lo:hi]), np_bits(y[lo:hi]),
+                         np_bits(p[lo // 32 * bits:(hi * bits + 31) // 32]).view(np.uint32), np_bits(gi[lo:hi]), f"c2 k={bits}"))
+        list(_POOL.map(lambda j: compare_block(*j), jobs))
+
+
+def test_config3_gelu_bf16_llm_ffn_sampled():
+    x, g = wl.draw(wl.C3, DEV)
+    assert x.numel() == 2 ** 28
+    for bits in wl.C3.bits:
+        y, p, gi = run_gpu("gelu", bits, x, g)
+        compare_sampled("gelu", bits, x, g, y, p, gi, f"c3 k={bits}", blocks=48, seed=bits)
+        # properties that hold at any size: code histogram equals the count of x per interval
+        s, _ = table("gelu", bits).arrays()
+        edges = torch.tensor(s, device=DEV)
+        ref_hist = torch.bincount(torch.bucketize(x.float(), edges, right=False), minlength=1 << bits)
+        words = p.view(torch.int32)
+        hist = torch.zeros(1 << bits, dtype=torch.int64, device=DEV)
+        if 32 % bits == 0:
+            for sh in range(0, 32, bits):
+                hist += torch.bincount((words >> sh) & ((1 << bits) - 1), minlength=1 << bits)
+            assert torch.equal(hist, ref_hist)
+        del y, p, gi
+
+
+def test_config4_cnn_f32_sampled():
+    x, g = wl.draw(wl.C4, DEV)
+    for act in wl.C4.acts:
+        y, p, gi = run_gpu(act, 2, x, g)
+        compare_sampled(act, 2, x, g, y, p, gi, f"c4 {act}", blocks=48, seed=3)
+
+
+@pytest.mark.parametrize("n", [2 ** 16, 2 ** 20])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_config5_sweep_small_full(n, dtype):
+    case = next(c for c in wl.sweep_cases([n]) if c.dtype == dtype)
+    x, g = wl.draw(case, DEV)
+    for act in case.acts:
+        for bits in case.bits:
+            y, p, gi = run_gpu(act, bits, x, g)
+            compare_full(act, bits, x, g, y, p, gi, f"c5 {act} k={bits} n={n} {dtype}")
+
+
+@pytest.mark.parametrize("n", [2 ** 24, 2 ** 24 + 7, 2 ** 28])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_config5_sweep_large_sampled(n, dtype):
+    case = next(c for c in wl.sweep_cases([n]) if c.dtype == dtype)
+    x, g = wl.draw(case, DEV)
+    blocks = 12 if n < 2 ** 28 else 8
+    for act in case.acts:
+        for bits in case.bits:
+            y, p, gi = run_gpu(act, bits, x, g)
+            compare_sampled(act, bits, x, g, y, p, gi, f"c5 {act} k={bits} n={n} {dtype}", blocks=blocks,
+                            block_elems=4096, seed=bits)
+            del y, p, gi
+
+
+# --------------------------------------------------------------------------
+# edge cases
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+def test_ragged_sizes(dtype, bits):
+    gen = torch.Generator(device=DEV).manual_seed(11)
+    for n in [1, 7, 31, 32, 33, 255, 256, 257, 1023, 1024, 1025, 2047, 2048 + 33, 5 * 1024 + 1000, 9999]:
+        x = (torch.randn(n, generator=gen, device=DEV) * 2).to(TORCH_DT[dtype])
+        g = torch.randn(n, generator=gen, device=DEV).to(TORCH_DT[dtype])
+        y, p, gi = run_gpu("silu", bits, x, g)
+        compare_full("silu", bits, x, g, y, p, gi, f"ragged n={n}")
+
+
+def test_empty_input_is_a_no_op():
+    t = table("gelu", 2)
+    x = torch.empty(0, device=DEV)
+    before = fb.fewbit_launch_count()
+    y, p = fb.fewbit_fwd(t, x)
+    gi = fb.fewbit_bwd(t, p, x)
+    assert y.numel() == 0 and p.numel() == 0 and gi.numel() == 0
+    assert fb.fewbit_launch_count() == before
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_in_place_aliasing(dtype):
+    gen = torch.Generator(device=DEV).manual_seed(5)
+    n = 70001
+    x = torch.randn(n, generator=gen, device=DEV).to(TORCH_DT[dtype])
+    g = torch.randn(n, generator=gen, device=DEV).to(TORCH_DT[dtype])
+    for bits in (1, 3):
+        y, p, gi = run_gpu("tanh", bits, x, g, inplace=True)
+        compare_full("tanh", bits, x, g, y, p, gi, "in place")
+
+
+@pytest.mark.parametrize("act", wl.ACTIVATIONS)
+def test_every_bf16_pattern(act):
+    """All 65 536 bfloat16 inputs: codes for every pattern (NaN and infinities
+    included), y for every finite input."""
+    h = torch.arange(65536, dtype=torch.int32).to(torch.int16).view(torch.bfloat16).to(DEV)
+    g = torch.ones_like(h)
+    for bits in (1, 4):
+        y, p, gi = run_gpu(act, bits, h, g)
+        compare_full(act, bits, h, g, y, p, gi, f"all bf16 {act}")
+
+
+@pytest.mark.parametrize("act", wl.ACTIVATIONS)
+def test_f32_values_around_every_boundary_and_in_the_tails(act):
+    pieces = []
+    for bits in (1, 2, 3, 4):
+        s, _ = table(act, bits).arrays()
+        pieces += [s, np.nextafter(s, np.float32(np.inf)), np.nextafter(s, np.float32(-np.inf))]
+    rng = np.random.default_rng(7)
+    mags = (10.0 ** rng.uniform(-44, 2.2, 20000)).astype(np.float32)
+    pieces += [mags, -mags, np.linspace(-20, 20, 40001, dtype=np.float32),
+               np.array([0.0, -0.0, 1e-45, -1e-45, 88.0, -88.0, 100.0, -100.0, -103.9, 3e38, -3e38], dtype=np.float32)]
+    x_np = np.concatenate(pieces)
+    x = torch.from_numpy(x_np).to(DEV)
+    g = torch.ones_like(x)
+    for bits in (1, 2, 3, 4):
+        y, p, gi = run_gpu(act, bits, x, g)
+        compare_full(act, bits, x, g, y, p, gi, f"special f32 {act} k={bits}")
+
+
+def test_gradient_specials_are_bit_exact():
+    """Denormal, huge and signed-zero gradients: one binary32 multiply, one rounding."""
+    rng = np.random.default_rng(3)
+    n = 40000
+    gf = (rng.standard_normal(n) * 10.0 ** rng.uniform(-44, 37, n)).astype(np.float32)
+    gf[:4] = [0.0, -0.0, 1e-45, -1e-45]
+    x = torch.from_numpy((rng.standard_normal(n) * 2).astype(np.float32)).to(DEV)
+    for dtype in ("f32", "bf16"):
+        g = torch.from_numpy(gf).to(DEV).to(TORCH_DT[dtype])
+        xs = x.to(TORCH_DT[dtype])
+        for bits in (2, 4):
+            y, p, gi = run_gpu("gelu", bits, xs, g)
+            compare_full("gelu", bits, xs, g, y, p, gi, f"grad specials {dtype}")
+
+
+def test_injected_table_with_equal_boundaries():
+    s = np.array([-1.0, 0.0, 0.0, 0.0, 0.5, 0.5, 3.0], dtype=np.float32)
+    lev = np.linspace(-1, 1, 8).astype(np.float32)
+    t = fb.fewbit_table_from_arrays("elu", 3, s, lev)
+    x = torch.linspace(-4, 4, 8193, device=DEV)
+    g = torch.ones_like(x)
+    y, p = fb.fewbit_fwd(t, x)
+    gi = fb.fewbit_bwd(t, p, g)
+    torch.cuda.synchronize()
+    y_ref, p_ref = oracle.fwd("elu", 3, s, np_bits(x))
+    gi_ref = oracle.bwd(3, lev, p_ref, np_bits(g))
+    assert np.array_equal(np_bits(p).view(np.uint32), p_ref)
+    assert np.array_equal(np_bits(gi), gi_ref)
+
+
+def test_misaligned_device_buffers_are_rejected():
+    t = table("gelu", 2)
+    x = torch.zeros(4096 + 8, device=DEV)
+    with pytest.raises(fb.FewbitError) as e:
+        fb.fewbit_fwd(t, x[1:4097])
+    assert e.value.status == 3
+
+
+def test_runs_on_a_side_stream():
+    t = table("silu", 4)
+    x = torch.randn(1 << 20, device=DEV).bfloat16()
+    g = torch.randn(1 << 20, device=DEV).bfloat16()
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        y, p = fb.fewbit_fwd(t, x)
+        gi = fb.fewbit_bwd(t, p, g)
+    st.synchronize()
+    compare_full("silu", 4, x, g, y, p, gi, "side stream")
+
+
+# --------------------------------------------------------------------------
+# host-buffer entry points
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_entry_points_match_the_oracle(dtype, pinned):
+    n = 300000 + 77
+    gen = torch.Generator().manual_seed(9)
+    x = torch.randn(n, generator=gen).to(TORCH_DT[dtype])
+    g = torch.randn(n, generator=gen).to(TORCH_DT[dtype])
+    if pinned:
+        x, g = x.pin_memory(), g.pin_memory()
+    for bits in (1, 3, 4):
+        t = table("softplus", bits)
+        words = fb.fewbit_packed_bytes(n, bits) // 4
+        mk = (lambda *a, **k: torch.empty(*a, **k).pin_memory()) if pinned else torch.empty
+        y, gi, p = mk(n, dtype=x.dtype), mk(n, dtype=x.dtype), mk(words, dtype=torch.int32)
+        # a workspace for 32768-element chunks forces ten pipeline steps
+        ws = torch.empty(fb.fewbit_host_workspace_bytes(32768, x.dtype, bits), dtype=torch.uint8, device=DEV)
+        fb.fewbit_fwd_host(t, x, y, p, ws)
+        fb.fewbit_bwd_host(t, p, g, gi, ws)
+        compare_full("softplus", bits, x, g, y, p, gi, f"host {dtype} k={bits}")

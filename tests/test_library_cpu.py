@@ -1,0 +1,150 @@
+"""CPU-only checks of the library: it loads, exports what include/fewbit.h
+declares, its host solver agrees with the oracle, and its argument checks
+answer before anything touches a GPU."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2202_00441_b200 as fb
+from paper_2202_00441_b200 import build as fb_build
+from paper_2202_00441_b200.workloads import ACTIVATIONS
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    fb_build.build_library()
+    return fb.load_library()
+
+
+def test_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "fewbit.h")).read()
+    names = re.findall(r"FEWBIT_API[^;]*?\b(fewbit_\w+)\s*\(", header)
+    assert len(names) >= 14
+    for name in names:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    for code in range(6):
+        assert lib.fewbit_status_string(code)
+    assert lib.fewbit_status_string(99) == b"unknown status"
+
+
+def test_packed_bytes(lib):
+    for bits in (1, 2, 3, 4):
+        for n in (0, 1, 31, 32, 33, 1000, 2 ** 24 + 7, 2 ** 28):
+            assert fb.fewbit_packed_bytes(n, bits) == 4 * ((n * bits + 31) // 32)
+    assert fb.fewbit_packed_bytes(100, 0) == 0 and fb.fewbit_packed_bytes(100, 5) == 0
+
+
+@pytest.mark.parametrize("act", ACTIVATIONS)
+def test_solver_matches_oracle(lib, act):
+    """The library's DP (Eq. 7-9) and the oracle's are separate programmes;
+    they must reach the same optimum.  Smooth f': same boundaries, levels equal
+    after rounding to binary32 (up to 1 ulp).  LeakyReLU
+    (piecewise-constant f'): every zero-error table is optimal, so only the
+    objective and the induced function q are compared."""
+    for bits in (1, 2, 3, 4):
+        t = fb.fewbit_table_create(act, bits)
+        s, lev = t.arrays()
+        r = oracle.dp_solve(act, bits, -8.0, 8.0, 4096)
+        assert t.objective == pytest.approx(r["objective"], abs=1e-12)
+        if act == "leaky_relu":
+            probe = np.linspace(-7.99, 7.99, 4001)
+            q_lib = lev[np.searchsorted(s, probe.astype(np.float32), side="left")]
+            q_ref = r["lev"].astype(np.float32)[np.searchsorted(r["s"].astype(np.float32), probe.astype(np.float32), side="left")]
+            np.testing.assert_allclose(q_lib, q_ref, atol=1e-7)
+        else:
+            rs, rlev = r["s"].astype(np.float32), r["lev"].astype(np.float32)
+            if act in ("sigmoid", "tanh") and not np.array_equal(s, rs):
+                # even f': a table and its mirror image have the same error,
+                # rounding noise picks one; both are the optimum
+                rs, rlev = -rs[::-1], rlev[::-1]
+            np.testing.assert_array_equal(s, rs)
+            np.testing.assert_allclose(lev, rlev, rtol=2e-7, atol=1e-9)
+
+
+def test_solver_other_range_matches_oracle(lib):
+    t = fb.fewbit_table_create_ex("silu", 3, -10.0, 10.0, 1000)
+    r = oracle.dp_solve("silu", 3, -10.0, 10.0, 1000)
+    assert t.objective == pytest.approx(r["objective"], abs=1e-12)
+    np.testing.assert_allclose(t.arrays()[0], r["s"].astype(np.float32), rtol=1e-6)
+
+
+def test_table_from_arrays_round_trip_and_validation(lib):
+    s = np.array([-1.0, 0.5, 2.0], dtype=np.float32)
+    lev = np.array([0.0, 0.25, 0.75, 1.0], dtype=np.float32)
+    t = fb.fewbit_table_from_arrays("tanh", 2, s, lev)
+    s2, lev2 = t.arrays()
+    np.testing.assert_array_equal(s, s2)
+    np.testing.assert_array_equal(lev, lev2)
+    assert np.isnan(t.objective)
+    with pytest.raises(fb.FewbitError):
+        fb.fewbit_table_from_arrays("tanh", 2, s[::-1].copy(), lev)
+    with pytest.raises(fb.FewbitError):
+        fb.fewbit_table_from_arrays("tanh", 2, np.array([0, np.nan, 1], np.float32), lev)
+    # equal boundaries (a degenerate table) are allowed
+    fb.fewbit_table_from_arrays("tanh", 2, np.array([0, 0, 1], np.float32), lev)
+
+
+def test_invalid_table_requests(lib):
+    assert not lib.fewbit_table_create(0, 0)
+    assert not lib.fewbit_table_create(0, 5)
+    assert not lib.fewbit_table_create(7, 2)
+    assert not lib.fewbit_table_create(-1, 2)
+    out = ctypes.c_void_p()
+    assert lib.fewbit_table_create_ex(0, 2, 1.0, 1.0, 100, ctypes.byref(out)) == 1
+    assert lib.fewbit_table_create_ex(0, 2, -1.0, 1.0, 3, ctypes.byref(out)) == 1
+    assert lib.fewbit_table_create_ex(0, 2, -1.0, 1.0, 100, None) == 1
+    lib.fewbit_table_destroy(None)
+
+
+def test_hot_path_argument_checks_need_no_gpu(lib):
+    """NULL / misaligned / empty requests are answered on the host."""
+    t = fb.fewbit_table_create("gelu", 3)
+    h = t.handle
+    A = 1 << 20                      # a fake, well aligned "device address"; never dereferenced
+    assert lib.fewbit_fwd(None, A, A, A, 10, 0, None) == 1
+    assert lib.fewbit_fwd(h, A, A, A, 10, 7, None) == 1
+    assert lib.fewbit_fwd(h, None, A, A, 10, 0, None) == 1
+    assert lib.fewbit_fwd(h, A, None, A, 10, 0, None) == 1
+    assert lib.fewbit_fwd(h, A, A, None, 10, 0, None) == 1
+    assert lib.fewbit_fwd(h, A + 16, A, A, 10, 0, None) == 3
+    assert lib.fewbit_fwd(h, A, A + 8, A, 10, 1, None) == 3
+    assert lib.fewbit_fwd(h, A, A, A + 4, 10, 1, None) == 3
+    assert lib.fewbit_fwd(h, None, None, None, 0, 0, None) == 0
+    assert lib.fewbit_bwd(None, A, A, A, 10, 0, None) == 1
+    assert lib.fewbit_bwd(h, None, A, A, 10, 0, None) == 1
+    assert lib.fewbit_bwd(h, A, A + 2, A, 10, 1, None) == 3
+    assert lib.fewbit_bwd(h, A, A, A, 0, 1, None) == 0
+    assert lib.fewbit_fwd_host(h, A, A, A, 10, 0, None, 0) == 1
+    assert lib.fewbit_fwd_host(h, A, A, A, 10, 0, A, 16) == 5
+    assert lib.fewbit_bwd_host(h, A, A, A, 10, 0, A + 8, 1 << 20) == 3
+    assert lib.fewbit_fwd_host(h, A, A, A, 0, 0, None, 0) == 0
+
+
+def test_host_workspace_bytes(lib):
+    assert fb.fewbit_host_workspace_bytes(1, fb.binding.torch.float32, 3) == 3 * (2 * 4096 + 512)
+    assert fb.fewbit_host_workspace_bytes(1 << 20, fb.binding.torch.bfloat16, 4) == 3 * (2 * (2 << 20) + (1 << 19))
+    assert load_zero(lib) == 0
+
+
+def load_zero(lib):
+    return lib.fewbit_host_workspace_bytes(100, 0, 9)
+
+
+def test_memory_ratio_reproduces_the_papers_accounting():
+    """Appendix memory table: RoBERTa-base keeps 36.0 MB of pointwise-
+    nonlinearity inputs out of 219.6 MB of activations; at b bits those shrink
+    to b/32 of fp32, which gives the printed 16 / 15 / 15 / 14 % savings."""
+    nonlin, total = 36.0, 219.6
+    printed = {1: 16, 2: 15, 3: 15, 4: 14}
+    for bits, pct in printed.items():
+        saved = nonlin * (1 - fb.fewbit_packed_bytes(32, bits) / (32 * 4)) / total
+        assert round(100 * saved) == pct
