@@ -236,8 +236,8 @@ def run_ours(args, case: wl.Case, act: str):
     torch.cuda.set_device(dev)
     fb.load_library()
 
-    n = case.n
-    x, g = wl.draw(dataclass_replace_seed(case, case.seed + rank), dev)
+    n = args.elements or case.n
+    x, g = wl.draw(dataclass_replace_seed(case, case.seed + rank), dev, n=n)
     y, gi = torch.empty_like(x), torch.empty_like(g)
     tables = {b: fb.fewbit_table_create(act, b) for b in case.bits}
     packed = {b: torch.empty(fb.fewbit_packed_bytes(n, b) // 4, dtype=torch.int32, device=dev) for b in case.bits}
@@ -246,7 +246,6 @@ def run_ours(args, case: wl.Case, act: str):
     if footprint < 512 * 2 ** 20:            # smaller than a few L2s: flush between launches
         flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
 
-    launches = [("fwd", b) for b in case.bits] + [("bwd", b) for b in case.bits]
     order = [(kind, b) for b in case.bits for kind in ("fwd", "bwd")]
 
     def one_step(events=None):
@@ -354,7 +353,8 @@ def run_ours(args, case: wl.Case, act: str):
             "metric": METRIC, "value": value, "unit": "elements/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": case.dtype, "data": "synthetic",
-            "config": {"workload": case.name, "act": act, "bits": list(case.bits), "shape": list(case.shape),
+            "config": {"workload": case.name if not args.elements else f"{case.name} cut to {n} elements",
+                       "act": act, "bits": list(case.bits), "shape": list(case.shape) if not args.elements else [n],
                        "elements": n, "launches_per_step": len(order),
                        "l2": "inputs larger than L2 (no flush)" if flush is None else "256 MiB flush write before every launch; value sums the launches",
                        "elements_counted": "once per kernel pass (forward and backward each count n)",
@@ -440,9 +440,11 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(wl.CONFIGS), default="c3")
     ap.add_argument("--act", default=None, help="activation of the workload to time (default: its first)")
+    ap.add_argument("--elements", type=int, default=0,
+                    help="draw only this many elements of the workload's distribution (small cases for profiling)")
     ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--cpu-sample", type=int, default=1 << 23)
-    ap.add_argument("--ref-sample", type=int, default=1 << 22)
+    ap.add_argument("--cpu-sample", type=int, default=1 << 26)
+    ap.add_argument("--ref-sample", type=int, default=1 << 25)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-torch-baseline", action="store_true")

@@ -12,7 +12,10 @@ INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "libfewbit.so")
 OBJ_DIR = os.path.join(PKG, "build")
 
-SOURCES = ["fewbit_kernels.cu", "fewbit_host.cu", "fewbit_table.cpp"]
+# (source, object stem, extra flags); the forward kernels are instantiated once per activation
+SOURCES = [("fewbit_kernels.cu", "fewbit_kernels", []), ("fewbit_host.cu", "fewbit_host", []),
+           ("fewbit_table.cpp", "fewbit_table", [])]
+SOURCES += [("fewbit_fwd_inst.cu", f"fewbit_fwd_act{a}", [f"-DFEWBIT_ACT_ID={a}"]) for a in range(7)]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC,-fvisibility=hidden,-O2", "-I", INCLUDE, "-I", CSRC,
@@ -36,21 +39,21 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     headers.append(os.path.join(INCLUDE, "fewbit.h"))
     os.makedirs(OBJ_DIR, exist_ok=True)
     jobs = []
-    for src in SOURCES:
+    for src, stem, extra in SOURCES:
         path = os.path.join(CSRC, src)
-        obj = os.path.join(OBJ_DIR, os.path.splitext(src)[0] + ".o")
+        obj = os.path.join(OBJ_DIR, stem + ".o")
         if force or _stale(obj, [path] + headers):
-            cmd = [_nvcc(), *NVCC_FLAGS, "-c", path, "-o", obj]
+            cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", path, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)
-    with concurrent.futures.ThreadPoolExecutor(max_workers=max(1, len(jobs))) as pool:
+    with concurrent.futures.ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 4))) as pool:
         for res in pool.map(lambda c: subprocess.run(c, capture_output=True, text=True), jobs):
             if verbose and res.stderr:
                 print(res.stderr)
             if res.returncode != 0:
                 raise RuntimeError("nvcc failed:\n" + " ".join(res.args) + "\n" + res.stdout + res.stderr)
-    objs = [os.path.join(OBJ_DIR, os.path.splitext(s)[0] + ".o") for s in SOURCES]
+    objs = [os.path.join(OBJ_DIR, stem + ".o") for _, stem, _ in SOURCES]
     if force or jobs or _stale(LIB, objs):
         tmp = LIB + f".{os.getpid()}.tmp"
         subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs])

@@ -1,0 +1,359 @@
+// Forward half of Listing 1 for sm_100a: y = f(x), code = position of x among
+// the boundaries (Eq. 2), codes bit-packed into whole 32-bit words.
+//
+// A CTA of 512 threads owns a contiguous stretch of 16 * iters warp-blocks of
+// 1024 elements; warp w takes warp-blocks w, w + 16, ... of it (see
+// fewbit_device.cuh for the lane / tile / warp-block decomposition and the quad
+// transpose that turns per-lane code groups into whole words).  The hardware
+// block scheduler balances the CTAs over the SMs (two resident per SM).
+//
+// Bucketize (code = #{ j : s[j] < x }, Eq. 2) has three implementations, mixed
+// so that no single pipe of the SM saturates before HBM does:
+//   search   : branch-free binary search on one binary32 element (ALU pipe);
+//   packed   : bfloat16 only -- the same search on TWO elements per
+//              instruction with bf16x2 compares against boundaries rounded
+//              down to bfloat16 (exact: s < x <=> floor_bf16(s) < x for a
+//              bfloat16 x), threshold selection by bitwise masks;
+//   look-up  : the code is a step function of x, so it is read from a byte
+//              table in shared memory indexed by the top bits of the pattern:
+//                bfloat16 : 65 536 entries, one per pattern, the exact code;
+//                binary32 : 8 192 entries (sign, exponent, 4 mantissa bits);
+//                           an entry m is the smallest code in its cell and
+//                           code = m + (s[m] < x), one binary32 comparison; a
+//                           cell with two or more boundaries (or infinity next
+//                           to NaNs) is marked dense and the warp redoes that
+//                           tile by search.
+//              The table arrives run-length encoded as a kernel parameter (a
+//              few dozen runs) and is expanded by the CTA before streaming.
+//              Random indices cost ~3.3 shared-memory wavefronts per warp
+//              look-up, which is why bfloat16 uses it for only half of the
+//              elements and only at 4 bits.
+// LUT = false: no table (bfloat16: packed search; binary32: search).
+#pragma once
+
+#include <cstdlib>
+
+#include "fewbit_device.cuh"
+#include "fewbit_math.cuh"
+
+namespace fewbit {
+
+constexpr int kFwdThreads = 512;
+constexpr int kFwdCtasPerSm = 2;
+
+template <typename T> struct Raw;                 // the 8 elements of a lane-chunk as loaded
+template <> struct Raw<float> { float v[8]; };
+template <> struct Raw<__nv_bfloat16> { uint32_t v[4]; };
+
+__device__ __forceinline__ void load_raw(const float *p, Raw<float> &r) { load8(p, r.v); }
+__device__ __forceinline__ void load_raw(const __nv_bfloat16 *p, Raw<__nv_bfloat16> &r) {
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]) : "l"(p) : "memory");
+}
+__device__ __forceinline__ float elem(const Raw<float> &r, int e) { return r.v[e]; }
+__device__ __forceinline__ float elem(const Raw<__nv_bfloat16> &r, int e) {
+    return __uint_as_float((e & 1) ? (r.v[e >> 1] & 0xffff0000u) : (r.v[e >> 1] << 16));
+}
+__device__ __forceinline__ uint32_t pair_bits(const Raw<float> &, int) { return 0; }
+__device__ __forceinline__ uint32_t pair_bits(const Raw<__nv_bfloat16> &r, int e) { return r.v[e >> 1]; }   // elements e, e+1 (e even)
+__device__ __forceinline__ uint32_t cell(const Raw<float> &r, int e) { return __float_as_uint(r.v[e]) >> (32 - kCellBitsF32); }
+__device__ __forceinline__ uint32_t cell(const Raw<__nv_bfloat16> &r, int e) {
+    return (e & 1) ? (r.v[e >> 1] >> 16) : (r.v[e >> 1] & 0xffffu);
+}
+
+struct FwdSmem {
+    uint32_t runs[kMaxRuns + 1];     // start | value << 24, plus a sentinel run starting one past the last cell
+    uint32_t work[kMaxRuns + 1];     // [0] = count, then 16-cell groups that straddle a run boundary
+    float thr[kMaxLevels];           // the boundaries, for the binary32 one-comparison step
+};
+
+// Largest r with start(runs[r]) <= c.
+__device__ __forceinline__ uint32_t find_run(const uint32_t *runs, uint32_t count, uint32_t c) {
+    uint32_t lo = 0, hi = count;                    // invariant: start[lo] <= c < start[hi]
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if ((runs[mid] & 0xffffffu) <= c) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Expands the run-length table into `lut` (CELLS bytes of shared memory).
+template <int CELLS, int THREADS>
+__device__ __forceinline__ void expand_runs(const CodeRuns &enc, uint8_t *lut, FwdSmem &sm) {
+    const uint32_t count = enc.count;
+    for (uint32_t i = threadIdx.x; i <= count; i += THREADS) sm.runs[i] = (i < count) ? enc.run[i] : static_cast<uint32_t>(CELLS);
+    if (threadIdx.x == 0) sm.work[0] = 0;
+    __syncthreads();
+    // A warp owns a contiguous stretch of 16-cell groups; lane l takes groups l, l + 32, ... of it,
+    // so that the 128-bit stores of one instruction fall on consecutive addresses (no bank conflict).
+    constexpr int kGroups = CELLS / 16;             // 16 cells = one 128-bit shared store
+    constexpr int kWarps = THREADS / 32;
+    constexpr int kPerWarp = (kGroups + kWarps - 1) / kWarps;
+    constexpr int kPerLane = (kPerWarp + 31) / 32;
+    const uint32_t first = (threadIdx.x >> 5) * kPerWarp + (threadIdx.x & 31);
+    if (first < kGroups) {
+        uint32_t r = find_run(sm.runs, count, first * 16);
+#pragma unroll 1
+        for (int i = 0; i < kPerLane; ++i) {
+            const uint32_t g = first + 32 * i;
+            if (g >= kGroups || g >= ((threadIdx.x >> 5) + 1) * kPerWarp) break;
+            const uint32_t a = g * 16;
+            while ((sm.runs[r + 1] & 0xffffffu) <= a) ++r;
+            if ((sm.runs[r + 1] & 0xffffffu) >= a + 16) {
+                const uint32_t v = (sm.runs[r] >> 24) * 0x01010101u;
+                *reinterpret_cast<uint4 *>(lut + a) = make_uint4(v, v, v, v);
+            } else {
+                sm.work[1 + atomicAdd(&sm.work[0], 1u)] = g;      // at most one group per run start
+            }
+        }
+    }
+    __syncthreads();
+    const uint32_t todo = sm.work[0] * 16;
+    for (uint32_t i = threadIdx.x; i < todo; i += THREADS) {
+        const uint32_t c = sm.work[1 + (i >> 4)] * 16 + (i & 15);
+        lut[c] = static_cast<uint8_t>(sm.runs[find_run(sm.runs, count, c)] >> 24);
+    }
+    __syncthreads();
+}
+
+struct FwdParams {
+    Boundaries tb;
+    uint32_t sb2[kMaxLevels];        // boundaries rounded down to bfloat16, replicated in both halves
+    CodeRuns runs;
+};
+
+// ---------------------------------------------------------------------------
+// packed search: codes of the two bfloat16 elements of `x2`, low element in
+// bits 0..3, high element in bits 16..19
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t gt2(uint32_t a, uint32_t b) {          // per half: 0xffff if a > b (false for NaN)
+    uint32_t r;
+    asm("set.gt.u32.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t sel2(uint32_t m, uint32_t a, uint32_t b) { return (m & a) | (~m & b); }
+
+template <int BITS>
+__device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLevels], uint32_t x2) {
+    if constexpr (BITS == 1) {
+        return gt2(x2, S[0]) & 0x00010001u;
+    } else if constexpr (BITS == 2) {
+        const uint32_t m1 = gt2(x2, S[1]);
+        const uint32_t m0 = gt2(x2, sel2(m1, S[2], S[0]));
+        return (m1 & 0x00020002u) | (m0 & 0x00010001u);
+    } else if constexpr (BITS == 3) {
+        const uint32_t m2 = gt2(x2, S[3]);
+        const uint32_t m1 = gt2(x2, sel2(m2, S[5], S[1]));
+        const uint32_t m0 = gt2(x2, sel2(m1, sel2(m2, S[6], S[2]), sel2(m2, S[4], S[0])));
+        uint32_t c = m2 & 0x00040004u;
+        c |= m1 & 0x00020002u;
+        return c | (m0 & 0x00010001u);
+    } else {
+        const uint32_t m3 = gt2(x2, S[7]);
+        const uint32_t m2 = gt2(x2, sel2(m3, S[11], S[3]));
+        const uint32_t m1 = gt2(x2, sel2(m2, sel2(m3, S[13], S[5]), sel2(m3, S[9], S[1])));
+        const uint32_t e0 = sel2(m3, S[8], S[0]), e1 = sel2(m3, S[10], S[2]);
+        const uint32_t e2 = sel2(m3, S[12], S[4]), e3 = sel2(m3, S[14], S[6]);
+        const uint32_t m0 = gt2(x2, sel2(m1, sel2(m2, e3, e1), sel2(m2, e2, e0)));
+        uint32_t c = m3 & 0x00080008u;
+        c |= m2 & 0x00040004u;
+        c |= m1 & 0x00020002u;
+        return c | (m0 & 0x00010001u);
+    }
+}
+
+// bfloat16: how many of the four element pairs of a lane-chunk use the look-up table when the
+// kernel has one (the rest use the packed search)
+#ifndef FEWBIT_LUT_PAIRS_K3
+#define FEWBIT_LUT_PAIRS_K3 4
+#endif
+#ifndef FEWBIT_LUT_PAIRS_K4
+#define FEWBIT_LUT_PAIRS_K4 4
+#endif
+template <int BITS> struct Bf16LutPairs { static constexpr int value = BITS == 4 ? FEWBIT_LUT_PAIRS_K4 : (BITS == 3 ? FEWBIT_LUT_PAIRS_K3 : 0); };
+
+template <int ACT, int BITS, typename T, bool LUT>
+__global__ void __launch_bounds__(kFwdThreads, kFwdCtasPerSm)
+fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters) {
+    constexpr bool kIsBf16 = sizeof(T) == 2;
+    constexpr int kCells = kIsBf16 ? (1 << kCellBitsBf16) : (1 << kCellBitsF32);
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    uint8_t *lut = smem_raw;
+    const float *thr = reinterpret_cast<const FwdSmem *>(smem_raw + kCells)->thr;
+
+    const int lane = threadIdx.x & 31;
+    constexpr size_t warps = kFwdThreads / 32;                                   // stride between a warp's warp-blocks
+    const size_t cta_begin = static_cast<size_t>(blockIdx.x) * warps * iters;
+    const size_t warp0 = cta_begin + (threadIdx.x >> 5);
+    const size_t all_full = n / kWarpElems;
+    const size_t cta_end = cta_begin + warps * iters;
+    const size_t full = all_full < cta_end ? all_full : cta_end;                 // this CTA's warp-blocks are [cta_begin, full)
+
+    // Software pipeline: as soon as a tile of the current warp-block has been consumed, the same
+    // registers are reloaded with that tile of the warp's next warp-block, so four loads per lane
+    // stay in flight while the warp computes.
+    Raw<T> cur[kTilesPerWarp];
+    if (warp0 < full) {
+        const T *px = x + warp0 * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
+#pragma unroll
+        for (int t = 0; t < kTilesPerWarp; ++t) load_raw(px + t * kTileElems, cur[t]);
+    }
+    if constexpr (LUT) {                                            // expanded while the first loads are in flight
+        FwdSmem &sm = *reinterpret_cast<FwdSmem *>(smem_raw + kCells);
+        if (threadIdx.x < kMaxLevels) sm.thr[threadIdx.x] = prm.tb.s[threadIdx.x];
+        expand_runs<kCells, kFwdThreads>(prm.runs, lut, sm);
+    }
+    for (size_t wb = warp0; wb < full; wb += warps) {
+        const size_t base = wb * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
+        T *py = y + base;
+        const T *px_next = x + base + warps * kWarpElems;
+        const bool more = wb + warps < full;
+        uint32_t grp[4];
+#pragma unroll
+        for (int t = 0; t < kTilesPerWarp; ++t) {
+            float o[8];
+            uint32_t g = 0;
+            [[maybe_unused]] uint32_t dense = 0;
+            [[maybe_unused]] uint32_t pc[4];                        // bfloat16: codes of element pair i, low @0, high @16
+#pragma unroll
+            for (int e = 6; e >= 0; e -= 2) {                       // two neighbouring elements at a time
+                const float2 xv = make_float2(elem(cur[t], e), elem(cur[t], e + 1));
+                const float2 yv = activation2<ACT, T>(xv);
+                o[e] = yv.x;
+                o[e + 1] = yv.y;
+                if constexpr (kIsBf16) {
+                    if (LUT && (e / 2) < Bf16LutPairs<BITS>::value) {              // resolved at compile time (unrolled)
+                        pc[e / 2] = lut[cell(cur[t], e)] + (static_cast<uint32_t>(lut[cell(cur[t], e + 1)]) << 16);
+                    } else {
+                        pc[e / 2] = bucketize_bf16x2<BITS>(prm.sb2, pair_bits(cur[t], e));
+                    }
+                } else {
+                    uint32_t c0, c1;
+                    if constexpr (!LUT) {
+                        c0 = bucketize<BITS>(prm.tb, xv.x);
+                        c1 = bucketize<BITS>(prm.tb, xv.y);
+                    } else {
+                        const uint32_t m0 = lut[cell(cur[t], e)], m1 = lut[cell(cur[t], e + 1)];
+                        dense |= m0 | m1;
+                        c0 = (m0 & 15u) + (thr[m0 & 15u] < xv.x ? 1u : 0u);
+                        c1 = (m1 & 15u) + (thr[m1 & 15u] < xv.y ? 1u : 0u);
+                    }
+                    g = (((g << BITS) + c1) << BITS) + c0;
+                }
+            }
+            if constexpr (kIsBf16) {
+                // eight codes -> one 8*BITS-bit group: merge pairs two by two while the low and the
+                // high elements still sit in separate halves, then fold the high half next to the low
+                const uint32_t a01 = pc[0] + (pc[1] << (2 * BITS)), a23 = pc[2] + (pc[3] << (2 * BITS));
+                constexpr uint32_t kFold = (1u << BITS) - (1u << 16);               // hi * 2^16 -> hi * 2^BITS
+                const uint32_t b01 = a01 + (a01 >> 16) * kFold, b23 = a23 + (a23 >> 16) * kFold;
+                g = b01 + (b23 << (4 * BITS));
+            }
+            if constexpr (LUT && !kIsBf16) {
+                if (__any_sync(0xffffffffu, dense & 0x80u)) {        // a dense cell: redo this tile's codes by search
+                    g = 0;
+#pragma unroll
+                    for (int e = 7; e >= 0; --e) g = (g << BITS) + bucketize<BITS>(prm.tb, elem(cur[t], e));
+                }
+            }
+            grp[t] = g;
+            store8(py + t * kTileElems, o);
+            if (more) load_raw(px_next + t * kTileElems, cur[t]);
+        }
+        quad_transpose(grp, lane);
+        uint32_t w[BITS];
+        groups_to_words<BITS>(grp, w);
+        store_words<BITS>(packed + wb * (32 * BITS) + (lane & 3) * (8 * BITS) + (lane >> 2) * BITS, w);
+    }
+
+    // ragged tail: the warp whose sequence reaches the index of the last, partial warp-block; a lane
+    // owns 32 consecutive elements = BITS words
+    if ((n % kWarpElems) != 0 && all_full >= cta_begin && all_full < cta_end && (all_full - warp0) % warps == 0) {
+        const size_t full = all_full;
+        const size_t base = full * kWarpElems + static_cast<size_t>(lane) * 32;
+        uint32_t w[BITS + 1];
+#pragma unroll
+        for (int j = 0; j <= BITS; ++j) w[j] = 0;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            if (base + e < n) {
+                const float xv = load1(x + base + e);
+                store1(y + base + e, activation<ACT, T>(xv));
+                const uint32_t c = bucketize<BITS>(prm.tb, xv);
+                const int pos = e * BITS;
+                w[pos >> 5] |= c << (pos & 31);
+                if ((pos & 31) + BITS > 32) w[(pos >> 5) + 1] |= c >> (32 - (pos & 31));
+            }
+        }
+        const size_t total_words = (n * BITS + 31) / 32;
+        const size_t first = full * (32 * BITS) + static_cast<size_t>(lane) * BITS;
+#pragma unroll
+        for (int j = 0; j < BITS; ++j)
+            if (first + j < total_words) packed[first + j] = w[j];
+    }
+}
+
+template <typename T, bool LUT>
+constexpr size_t fwd_smem_bytes() {
+    return LUT ? (sizeof(T) == 2 ? (1u << kCellBitsBf16) : (1u << kCellBitsF32)) + sizeof(FwdSmem) : 0;
+}
+
+int device_sm_count(cudaError_t *err);   // of the current device, cached
+const char *fwd_iters_override();        // tuning aid: environment FEWBIT_FWD_ITERS
+
+template <int ACT, int BITS, typename T, bool LUT>
+cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *packed, size_t n, cudaStream_t st) {
+    cudaError_t err = cudaSuccess;
+    const int sms = device_sm_count(&err);
+    if (err != cudaSuccess) return err;
+    constexpr size_t smem = fwd_smem_bytes<T, LUT>();
+    auto kernel = fwd_kernel<ACT, BITS, T, LUT>;
+    if constexpr (smem > 48 * 1024) {
+        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (err != cudaSuccess) return err;
+    }
+    constexpr size_t warps_per_cta = kFwdThreads / 32;
+    const size_t warp_blocks = n / kWarpElems + ((n % kWarpElems) ? 1 : 0);
+    // Iterations per warp.  Without a table: short CTAs, ~6 waves over the resident slots (the
+    // block scheduler evens out SMs that run slow), at most 8.  With a table the expansion has to
+    // be amortised: ~2 waves, at most 32.
+    constexpr size_t kMaxIters = LUT ? 32 : 8;
+    constexpr size_t kWaves = LUT ? 2 : 6;
+    const size_t slots = static_cast<size_t>(sms) * kFwdCtasPerSm;
+    size_t iters = warp_blocks / (warps_per_cta * slots * kWaves);
+    iters = iters < 1 ? 1 : (iters > kMaxIters ? kMaxIters : iters);
+    if (const char *dbg = fwd_iters_override()) iters = static_cast<size_t>(atoi(dbg));
+    const size_t per_cta = warps_per_cta * iters;
+    const unsigned grid = static_cast<unsigned>((warp_blocks + per_cta - 1) / per_cta);
+    kernel<<<grid, kFwdThreads, smem, st>>>(prm, static_cast<const T *>(x), static_cast<T *>(y), packed, n,
+                                             static_cast<int>(iters));
+    return cudaGetLastError();
+}
+
+using FwdLaunch = cudaError_t (*)(const FwdParams &, const void *, void *, uint32_t *, size_t, cudaStream_t);
+
+// Launchers of one activation: [bits - 1][dtype is bf16][use look-up table]
+struct FwdLaunchers { FwdLaunch fn[kMaxBits][2][2]; };
+
+template <int ACT, int BITS>
+constexpr void fill_fwd_launchers(FwdLaunchers &l) {
+    l.fn[BITS - 1][0][0] = launch_fwd<ACT, BITS, float, false>;
+    // 1-2 bit binary32 tables: the search is 1-3 comparisons, cheaper than the table
+    l.fn[BITS - 1][0][1] = BITS >= 3 ? launch_fwd<ACT, BITS, float, (BITS >= 3)> : launch_fwd<ACT, BITS, float, false>;
+    l.fn[BITS - 1][1][0] = launch_fwd<ACT, BITS, __nv_bfloat16, false>;
+    l.fn[BITS - 1][1][1] = launch_fwd<ACT, BITS, __nv_bfloat16, (Bf16LutPairs<BITS>::value > 0)>;
+}
+
+template <int ACT>
+FwdLaunchers make_fwd_launchers() {
+    FwdLaunchers l{};
+    fill_fwd_launchers<ACT, 1>(l);
+    fill_fwd_launchers<ACT, 2>(l);
+    fill_fwd_launchers<ACT, 3>(l);
+    fill_fwd_launchers<ACT, 4>(l);
+    return l;
+}
+
+const FwdLaunchers &fwd_launchers(int act);   // defined by the per-activation translation units
+
+}  // namespace fewbit

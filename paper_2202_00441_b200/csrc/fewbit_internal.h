@@ -15,6 +15,31 @@ extern std::atomic<uint64_t> g_launches;     // kernels launched by the library 
 extern thread_local int t_last_cuda_error;   // cudaError_t behind this thread's last FEWBIT_ERR_CUDA
 }  // namespace fewbit
 
+namespace fewbit {
+
+// Run-length form of a code look-up table over the top bits of an element's
+// bit pattern ("cells").  Run i covers cells [start_i, start_{i+1}) and holds
+// one byte value; entry = start | value << 24.  The forward kernel expands it
+// into shared memory.
+//   bf16 table: one cell per bfloat16 pattern (65 536 cells), value = code.
+//   fp32 table: one cell per top-13-bit pattern (8 192 cells), value = the
+//               smallest code m in the cell when the cell holds at most one
+//               boundary (then code(x) = m + (s[m] < x)), else kCellDense.
+constexpr int kMaxRuns = 120;
+constexpr int kCellBitsBf16 = 16;
+constexpr int kCellBitsF32 = 13;
+constexpr unsigned kCellDense = 0xffu;
+
+struct CodeRuns {
+    uint32_t count;                    // 0: table not expressible, use the search kernel
+    uint32_t run[kMaxRuns];
+};
+
+void build_code_runs(const float *s, int bits, CodeRuns *bf16_runs, CodeRuns *f32_runs);
+void build_bf16_thresholds(const float *s, uint32_t *s_bf16x2);
+
+}  // namespace fewbit
+
 // The parameters s and y of Eq. 2, as binary32.  Unused boundary slots hold
 // +inf (never below any x), unused level slots 0.
 struct fewbit_table {
@@ -23,4 +48,7 @@ struct fewbit_table {
     double objective;                  // value of Eq. 3 reached by the solver
     float s[fewbit::kMaxLevels];       // s[0 .. K-2]
     float lev[fewbit::kMaxLevels];     // lev[0 .. K-1]
+    uint32_t s_bf16x2[fewbit::kMaxLevels];   // derived from s: largest bfloat16 <= s[j], in both halves of a word
+    fewbit::CodeRuns runs_bf16;        // derived from s: the bucketize step as a look-up table
+    fewbit::CodeRuns runs_f32;
 };

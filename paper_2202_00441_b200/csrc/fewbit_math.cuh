@@ -1,10 +1,21 @@
-// Device evaluation of the activations f (Sec. 2).  activation<ACT, T>(x)
-// returns f(x) as a binary32 value that the caller rounds to the storage type
-// T.  The result must stay within 2 ulp of T from the exactly rounded value:
-//   T = float    : evaluated in binary64 (errors far below a binary32 ulp);
-//   T = bfloat16 : evaluated in binary32 (errors far below a bfloat16 ulp),
-//                  in forms that keep RELATIVE accuracy in the tails, since
-//                  bfloat16 has the exponent range of binary32.
+// Device evaluation of the activations f (Sec. 2).
+//
+// activation<ACT, T>(x) returns f(x) as a binary32 value that the caller
+// rounds once (nearest-even) to the storage type T.  The rounded result must
+// stay within 2 ulp of T from the correctly rounded value, over the whole
+// input range -- including the tails, where f(x) is tiny but still a normal
+// number of T (bfloat16 has the exponent range of binary32).
+//
+//   T = bfloat16 : binary32 arithmetic with hardware approximations (ex2, rcp,
+//                  lg2, tanh: relative error <= 2^-11, far below the 2^-9 that
+//                  one bfloat16 ulp allows).  Every form is written so that
+//                  the small quantity is computed as a product, never as a
+//                  difference of nearly equal numbers:
+//                      e^{-|x|} and friends are produced as E * 2^64 (so that
+//                      ex2.approx.ftz never flushes them) and the factor
+//                      2^-64 is folded into the last fused multiply-add, whose
+//                      IEEE gradual underflow gives correct subnormals.
+//   T = float    : binary64 arithmetic (errors far below a binary32 ulp).
 #pragma once
 
 #include <cuda_bf16.h>
@@ -13,7 +24,85 @@
 
 namespace fewbit {
 
-// ---- binary64 evaluation (T = float) ---------------------------------------
+// ---- hardware approximations ------------------------------------------------
+__device__ __forceinline__ float ex2_ftz(float a) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a)); return r; }
+__device__ __forceinline__ float rcp_ftz(float a) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a)); return r; }
+__device__ __forceinline__ float lg2_ftz(float a) { float r; asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a)); return r; }
+__device__ __forceinline__ float tanh_apx(float a) { float r; asm("tanh.approx.f32 %0, %1;" : "=f"(r) : "f"(a)); return r; }
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kScaleUp = 64.0f;                      // exponent offset S
+constexpr float kScaleDown = 5.421010862427522e-20f;   // 2^-64
+
+// ---- packed binary32 pairs (sm_100: two FMAs per issued instruction) ----------
+__device__ __forceinline__ float2 splat(float c) { return make_float2(c, c); }
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ float2 relu2(float2 x) { return make_float2(fmaxf(x.x, 0.0f), fmaxf(x.y, 0.0f)); }
+// |x| = 2 max(x,0) - x, exact
+__device__ __forceinline__ float2 abs2_from_relu(float2 relu, float2 x) { return fma2(relu, splat(2.0f), make_float2(-x.x, -x.y)); }
+__device__ __forceinline__ float2 ex2_2(float2 a) { return make_float2(ex2_ftz(a.x), ex2_ftz(a.y)); }
+__device__ __forceinline__ float2 rcp_2(float2 a) { return make_float2(rcp_ftz(a.x), rcp_ftz(a.y)); }
+
+// ---- binary32 evaluation for bfloat16 storage, two elements at a time ---------
+template <int ACT>
+__device__ __forceinline__ float2 act_bf16(float2 x) {
+    if constexpr (ACT == FEWBIT_GELU) {
+        // x Phi(x) = max(x,0) - t Phi(-t), t = |x|, and
+        // t Phi(-t) = t e^{-t^2/2} G(w), w = 1/(1 + p t): G is a cubic times w fitted to
+        // Phi(-t) e^{t^2/2} on [0, 14.5] with relative error 2.3e-4 (the fit is
+        // paper_2202_00441_b200/csrc/fit_coefficients.py)
+        const float2 relu = relu2(x);
+        const float2 t = abs2_from_relu(relu, x);
+        const float2 e = ex2_2(fma2(mul2(x, x), splat(-0.5f * kLog2e), splat(kScaleUp)));
+        const float2 w = rcp_2(fma2(t, splat(0.30f), splat(1.0f)));
+        float2 g = fma2(w, splat(0.20884148f), splat(0.03559305f));
+        g = fma2(g, w, splat(0.13747554f));
+        g = fma2(g, w, splat(0.11820479f));
+        const float2 q = mul2(mul2(g, w), e);
+        return fma2(mul2(t, q), splat(-kScaleDown), relu);
+    } else if constexpr (ACT == FEWBIT_SILU) {
+        // x sigmoid(x) = max(x,0) - |x| E / (1 + E)
+        const float2 relu = relu2(x);
+        const float2 t = abs2_from_relu(relu, x);
+        const float2 e = ex2_2(fma2(t, splat(-kLog2e), splat(kScaleUp)));
+        const float2 r = rcp_2(fma2(e, splat(kScaleDown), splat(1.0f)));
+        return fma2(mul2(mul2(t, e), r), splat(-kScaleDown), relu);
+    } else if constexpr (ACT == FEWBIT_SIGMOID) {
+        // x >= 0: 1 - E/(1+E);  x < 0: E/(1+E)
+        const float2 step = make_float2(x.x >= 0.0f ? 1.0f : 0.0f, x.y >= 0.0f ? 1.0f : 0.0f);
+        const float2 e = ex2_2(make_float2(fmaf(fabsf(x.x), -kLog2e, kScaleUp), fmaf(fabsf(x.y), -kLog2e, kScaleUp)));
+        const float2 q = mul2(e, rcp_2(fma2(e, splat(kScaleDown), splat(1.0f))));
+        const float2 sgn = fma2(step, splat(-2.0f), splat(1.0f));
+        return fma2(mul2(q, sgn), splat(kScaleDown), step);
+    } else if constexpr (ACT == FEWBIT_TANH) {
+        return make_float2(tanh_apx(x.x), tanh_apx(x.y));
+    } else if constexpr (ACT == FEWBIT_ELU) {
+        // e^x - 1 = 2u / (1 - u), u = tanh(x/2): no cancellation for x <= 0
+        const float2 h = mul2(x, splat(0.5f));
+        const float2 u = make_float2(tanh_apx(h.x), tanh_apx(h.y));
+        const float2 m = mul2(add2(u, u), rcp_2(fma2(u, splat(-1.0f), splat(1.0f))));
+        return make_float2(x.x > 0.0f ? x.x : m.x, x.y > 0.0f ? x.y : m.y);
+    } else if constexpr (ACT == FEWBIT_SOFTPLUS) {
+        // max(x,0) + log(1 + E); for small E the logarithm is E (1 - E/2 + E^2/3) to keep relative accuracy
+        const float2 relu = relu2(x);
+        const float2 t = abs2_from_relu(relu, x);
+        const float2 e = ex2_2(fma2(t, splat(-kLog2e), splat(kScaleUp)));
+        const float2 es = mul2(e, splat(kScaleDown));                  // E; may underflow, only used while E is large
+        const float2 one_es = add2(es, splat(1.0f));
+        const float2 big = mul2(make_float2(lg2_ftz(one_es.x), lg2_ftz(one_es.y)), splat(kLn2 * 18446744073709551616.0f));
+        const float2 small = mul2(e, fma2(es, fma2(es, splat(0.33333334f), splat(-0.5f)), splat(1.0f)));
+        const float2 l = make_float2(es.x < 0.0625f ? small.x : big.x, es.y < 0.0625f ? small.y : big.y);
+        return fma2(l, splat(kScaleDown), relu);
+    } else {
+        const float2 m = mul2(x, splat(0.01f));
+        return make_float2(fmaxf(x.x, m.x), fmaxf(x.y, m.y));
+    }
+}
+
+// ---- binary64 evaluation for binary32 storage --------------------------------
 template <int ACT>
 __device__ __forceinline__ float act_f64(float xf) {
     const double x = static_cast<double>(xf);
@@ -38,32 +127,14 @@ __device__ __forceinline__ float act_f64(float xf) {
     return static_cast<float>(r);
 }
 
-// ---- binary32 evaluation (T = bfloat16) ------------------------------------
-template <int ACT>
-__device__ __forceinline__ float act_f32(float x) {
-    if constexpr (ACT == FEWBIT_GELU) {
-        return 0.5f * x * erfcf(-x * 0.70710678f);
-    } else if constexpr (ACT == FEWBIT_SILU) {
-        const float e = expf(-fabsf(x));
-        return (x >= 0.0f ? x : x * e) / (1.0f + e);
-    } else if constexpr (ACT == FEWBIT_SIGMOID) {
-        const float e = expf(-fabsf(x));
-        return (x >= 0.0f ? 1.0f : e) / (1.0f + e);
-    } else if constexpr (ACT == FEWBIT_TANH) {
-        return tanhf(x);
-    } else if constexpr (ACT == FEWBIT_ELU) {
-        return x > 0.0f ? x : expm1f(x);
-    } else if constexpr (ACT == FEWBIT_SOFTPLUS) {
-        return fmaxf(x, 0.0f) + log1pf(expf(-fabsf(x)));
-    } else {
-        return x > 0.0f ? x : 0.01f * x;
-    }
+// two neighbouring elements at once
+template <int ACT, typename T>
+__device__ __forceinline__ float2 activation2(float2 x) {
+    if constexpr (sizeof(T) == 4) return make_float2(act_f64<ACT>(x.x), act_f64<ACT>(x.y));
+    else return act_bf16<ACT>(x);
 }
 
 template <int ACT, typename T>
-__device__ __forceinline__ float activation(float x) {
-    if constexpr (sizeof(T) == 4) return act_f64<ACT>(x);
-    else return act_f32<ACT>(x);
-}
+__device__ __forceinline__ float activation(float x) { return activation2<ACT, T>(make_float2(x, x)).x; }
 
 }  // namespace fewbit

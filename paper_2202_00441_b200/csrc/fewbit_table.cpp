@@ -144,10 +144,68 @@ std::shared_ptr<const Solved> solved_for(fewbit_act act, double A, double B, int
     return g_cache.emplace(key, fresh).first->second;
 }
 
+// code(x) = #{ j : s[j] < x } by a plain scan (host side, table set-up only)
+inline unsigned code_of(const float *s, int nb, float x) {
+    unsigned c = 0;
+    for (int j = 0; j < nb; ++j) c += (s[j] < x) ? 1u : 0u;
+    return c;
+}
+
+inline float from_bits(uint32_t u) { float f; std::memcpy(&f, &u, 4); return f; }
+
+void encode_runs(const std::vector<uint8_t> &lut, CodeRuns *out) {
+    out->count = 0;
+    for (size_t c = 0; c < lut.size(); ++c) {
+        if (c == 0 || lut[c] != lut[c - 1]) {
+            if (out->count == kMaxRuns) { out->count = 0; return; }     // too fragmented: no look-up table
+            out->run[out->count++] = static_cast<uint32_t>(c) | (static_cast<uint32_t>(lut[c]) << 24);
+        }
+    }
+}
+
 bool valid_act(int a) { return a >= 0 && a < FEWBIT_NUM_ACTS; }
 bool valid_bits(int b) { return b >= 1 && b <= 4; }
 
 }  // namespace
+
+// Eq. 2's interval search as a table over bit patterns: the code is a step
+// function of x with at most K-1 steps, so it is constant on long runs of
+// patterns.
+void build_code_runs(const float *s, int bits, CodeRuns *bf16_runs, CodeRuns *f32_runs) {
+    const int nb = (1 << bits) - 1;
+    {   // bfloat16: exact code of every one of the 65 536 patterns
+        std::vector<uint8_t> lut(1u << kCellBitsBf16);
+        for (uint32_t p = 0; p < lut.size(); ++p) lut[p] = static_cast<uint8_t>(code_of(s, nb, from_bits(p << 16)));
+        encode_runs(lut, bf16_runs);
+    }
+    {   // binary32: per cell of 2^19 consecutive patterns, the smaller of the codes of its two
+        // end points when they differ by at most one (codes are monotone across a cell)
+        std::vector<uint8_t> lut(1u << kCellBitsF32);
+        const int shift = 32 - kCellBitsF32;
+        for (uint32_t p = 0; p < lut.size(); ++p) {
+            const unsigned a = code_of(s, nb, from_bits(p << shift));
+            const unsigned b = code_of(s, nb, from_bits((p << shift) | ((1u << shift) - 1u)));
+            const unsigned lo = a < b ? a : b, hi = a < b ? b : a;
+            // a cell that mixes infinity with NaNs (code 0) is dense unless K-1 <= 1
+            lut[p] = static_cast<uint8_t>((hi - lo <= 1) ? lo : kCellDense);
+        }
+        encode_runs(lut, f32_runs);
+    }
+}
+
+// For a bfloat16 x and any binary32 s:  s < x  <=>  floor_bf16(s) < x, where floor_bf16(s) is the
+// largest bfloat16 not above s.  The forward kernel compares two bfloat16 elements per instruction
+// against these rounded-down boundaries.
+void build_bf16_thresholds(const float *s, uint32_t *s_bf16x2) {
+    for (int j = 0; j < kMaxLevels; ++j) {
+        uint32_t u;
+        std::memcpy(&u, &s[j], 4);
+        uint32_t h = u >> 16;
+        if ((u & 0xffffu) != 0 && (u >> 31) != 0 && !std::isnan(s[j])) h += 1;   // negative and inexact: one step further from zero
+        s_bf16x2[j] = h | (h << 16);
+    }
+}
+
 }  // namespace fewbit
 
 using fewbit::kMaxLevels;
@@ -179,6 +237,8 @@ fewbit_status fewbit_table_create_ex(fewbit_act act, int bits, double A, double 
             t->s[m - 1] = static_cast<float>(sm);
         }
         for (int m = 0; m < K; ++m) t->lev[m] = static_cast<float>(g->level(ends[m], ends[m + 1]));   // Eq. 4
+        fewbit::build_code_runs(t->s, bits, &t->runs_bf16, &t->runs_f32);
+        fewbit::build_bf16_thresholds(t->s, t->s_bf16x2);
         *out = t;
         return FEWBIT_OK;
     } catch (const std::bad_alloc &) {
@@ -214,6 +274,8 @@ fewbit_status fewbit_table_from_arrays(fewbit_act act, int bits, const float *s,
     // +0 and -0 compare equal; store +0 so that every kernel variant sees one pattern
     for (int m = 0; m < K - 1; ++m) t->s[m] = (s[m] == 0.0f) ? 0.0f : s[m];
     for (int m = 0; m < K; ++m) t->lev[m] = lev[m];
+    fewbit::build_code_runs(t->s, bits, &t->runs_bf16, &t->runs_f32);
+    fewbit::build_bf16_thresholds(t->s, t->s_bf16x2);
     *out = t;
     return FEWBIT_OK;
 }
