@@ -38,7 +38,9 @@
 
 namespace fewbit {
 
-constexpr int kFwdThreads = 512;
+// threads per CTA: binary32 keeps 32 registers of input in flight per thread, so it runs fewer,
+// fatter threads (register cap 80) than bfloat16 (cap 64)
+template <typename T> struct FwdThreads { static constexpr int value = sizeof(T) == 2 ? 512 : 384; };
 constexpr int kFwdCtasPerSm = 2;
 
 template <typename T> struct Raw;                 // the 8 elements of a lane-chunk as loaded
@@ -173,9 +175,10 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
 template <int BITS> struct Bf16LutPairs { static constexpr int value = BITS == 4 ? FEWBIT_LUT_PAIRS_K4 : (BITS == 3 ? FEWBIT_LUT_PAIRS_K3 : 0); };
 
 template <int ACT, int BITS, typename T, bool LUT>
-__global__ void __launch_bounds__(kFwdThreads, kFwdCtasPerSm)
+__global__ void __launch_bounds__(FwdThreads<T>::value, kFwdCtasPerSm)
 fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters) {
     constexpr bool kIsBf16 = sizeof(T) == 2;
+    constexpr int kFwdThreads = FwdThreads<T>::value;
     constexpr int kCells = kIsBf16 ? (1 << kCellBitsBf16) : (1 << kCellBitsF32);
     extern __shared__ __align__(16) uint8_t smem_raw[];
     uint8_t *lut = smem_raw;
@@ -312,6 +315,7 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
         err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (err != cudaSuccess) return err;
     }
+    constexpr int kFwdThreads = FwdThreads<T>::value;
     constexpr size_t warps_per_cta = kFwdThreads / 32;
     const size_t warp_blocks = n / kWarpElems + ((n % kWarpElems) ? 1 : 0);
     // Iterations per warp.  Without a table: short CTAs, ~6 waves over the resident slots (the

@@ -15,7 +15,8 @@
 //                      ex2.approx.ftz never flushes them) and the factor
 //                      2^-64 is folded into the last fused multiply-add, whose
 //                      IEEE gradual underflow gives correct subnormals.
-//   T = float    : binary64 arithmetic (errors far below a binary32 ulp).
+//   T = float    : binary32 arithmetic built on an exponential good to ~0.7 ulp
+//                  (GELU: binary64 arithmetic).
 #pragma once
 
 #include <cuda_bf16.h>
@@ -127,10 +128,102 @@ __device__ __forceinline__ float act_f64(float xf) {
     return static_cast<float>(r);
 }
 
+// ---- binary32 evaluation for binary32 storage, two elements at a time ---------
+// Everything that must be accurate to a fraction of a binary32 ulp is built on one
+// exponential with ~0.7 ulp error; the quotient E / (1 + E) is refined with the
+// exact rounding error of the sum 1 + E, so the logistic function ends near 1 ulp.
+
+// e^a = (1 + s) * 2^n for a <= 0 (a is clamped at -131, far below the last value that matters:
+// every result that uses it has reached its limit in binary32 by then).  Cody-Waite reduction by
+// ln 2 in two pieces, degree-6 polynomial (fit in fit_coefficients.py: 0.05 ulp).  Returns s; *t
+// holds 1.5 * 2^23 + n, i.e. the integer n in its low mantissa bits.
+__device__ __forceinline__ float2 exp_reduced_f32(float2 a, float2 *t_out) {
+    a = make_float2(fmaxf(a.x, -131.0f), fmaxf(a.y, -131.0f));
+    const float2 t = fma2(a, splat(kLog2e), splat(12582912.0f));
+    const float2 n = add2(t, splat(-12582912.0f));
+    float2 r = fma2(n, splat(-0.693145751953125f), a);                      // ln 2, high 12 bits
+    r = fma2(n, splat(-1.428606765330187e-06f), r);                         // ln 2, the rest
+    float2 q = fma2(r, splat(0.0013814608100801706f), splat(0.008368746377527714f));
+    q = fma2(q, r, splat(0.04166838899254799f));
+    q = fma2(q, r, splat(0.1666652113199234f));
+    q = fma2(q, r, splat(0.4999999403953552f));
+    *t_out = t;
+    return fma2(mul2(r, r), q, r);                                           // e^r - 1
+}
+
+// 2^(n + bias - 127) from t = 1.5 * 2^23 + n, with integers
+__device__ __forceinline__ float2 pow2_from_t(float2 t, uint32_t bias) {
+    return make_float2(__uint_as_float((__float_as_uint(t.x) << 23) + (bias << 23)),
+                       __uint_as_float((__float_as_uint(t.y) << 23) + (bias << 23)));
+}
+
+// E * 2^64 for E = e^a, a <= 0
+__device__ __forceinline__ float2 exp_scaled_f32(float2 a) {
+    float2 t;
+    const float2 s = exp_reduced_f32(a, &t);
+    return mul2(add2(s, splat(1.0f)), pow2_from_t(t, 127u + 64u));
+}
+
+// e^a - 1 for a <= 0:  2^n (1 + s) - 1 = 2^n s + (2^n - 1), and 2^n - 1 is exact.  The result is
+// -1 in binary32 long before a = -80, where a is clamped so that 2^n stays a normal number.
+__device__ __forceinline__ float2 expm1_nonpos_f32(float2 a) {
+    a = make_float2(fmaxf(a.x, -80.0f), fmaxf(a.y, -80.0f));
+    float2 t;
+    const float2 s = exp_reduced_f32(a, &t);
+    const float2 p2 = pow2_from_t(t, 127u);
+    return fma2(p2, s, add2(p2, splat(-1.0f)));
+}
+
+// -(E / (1 + E)) * 2^64 for E = e^{-|x|}: Newton-corrected quotient with the rounding error of
+// 1 + E taken into account (Dh + Dl = 1 + E exactly).
+__device__ __forceinline__ float2 neg_logistic_tail_scaled_f32(float2 x) {
+    const float2 es = exp_scaled_f32(make_float2(-fabsf(x.x), -fabsf(x.y)));
+    const float2 e = mul2(es, splat(kScaleDown));
+    const float2 dh = add2(e, splat(1.0f));
+    const float2 dl = fma2(add2(dh, splat(-1.0f)), splat(-1.0f), e);
+    const float2 rn = make_float2(rcp_ftz(-dh.x), rcp_ftz(-dh.y));           // -1 / Dh
+    const float2 qn = mul2(es, rn);                                          // -q0
+    float2 res = fma2(dh, qn, es);                                           // E - Dh q0
+    res = fma2(dl, qn, res);                                                 //   - Dl q0
+    return fma2(res, rn, qn);                                                // -(q0 + res / Dh)
+}
+
+template <int ACT>
+__device__ __forceinline__ float2 act_f32(float2 x) {
+    if constexpr (ACT == FEWBIT_SILU) {
+        // x < 0: x q;  x >= 0: x - x q   with q = E / (1 + E)
+        // below -131 the product is 0 in binary32; clamping there keeps |x| E from growing again
+        // once E itself has been clamped
+        const float2 xc = make_float2(fmaxf(x.x, -131.0f), fmaxf(x.y, -131.0f));
+        const float2 u = mul2(xc, neg_logistic_tail_scaled_f32(xc));         // -x q 2^64
+        const float2 c = make_float2(copysignf(kScaleDown, x.x), copysignf(kScaleDown, x.y));
+        return fma2(u, make_float2(c.x, c.y), relu2(x));
+    } else if constexpr (ACT == FEWBIT_SIGMOID) {
+        // x < 0: q;  x >= 0: 1 - q
+        const float2 qn = neg_logistic_tail_scaled_f32(x);
+        const float2 step = make_float2(x.x >= 0.0f ? 1.0f : 0.0f, x.y >= 0.0f ? 1.0f : 0.0f);
+        const float2 c = fma2(step, splat(2.0f * kScaleDown), splat(-kScaleDown));
+        return fma2(qn, c, step);
+    } else if constexpr (ACT == FEWBIT_TANH) {
+        return make_float2(tanhf(x.x), tanhf(x.y));                          // library: <= 2 ulp
+    } else if constexpr (ACT == FEWBIT_ELU) {
+        const float2 m = expm1_nonpos_f32(make_float2(fminf(x.x, 0.0f), fminf(x.y, 0.0f)));
+        return make_float2(x.x > 0.0f ? x.x : m.x, x.y > 0.0f ? x.y : m.y);
+    } else if constexpr (ACT == FEWBIT_SOFTPLUS) {
+        const float2 e = mul2(exp_scaled_f32(make_float2(-fabsf(x.x), -fabsf(x.y))), splat(kScaleDown));
+        return add2(relu2(x), make_float2(log1pf(e.x), log1pf(e.y)));
+    } else if constexpr (ACT == FEWBIT_LEAKY_RELU) {
+        const float2 m = mul2(x, splat(0.01f));
+        return make_float2(fmaxf(x.x, m.x), fmaxf(x.y, m.y));
+    } else {
+        return make_float2(act_f64<ACT>(x.x), act_f64<ACT>(x.y));
+    }
+}
+
 // two neighbouring elements at once
 template <int ACT, typename T>
 __device__ __forceinline__ float2 activation2(float2 x) {
-    if constexpr (sizeof(T) == 4) return make_float2(act_f64<ACT>(x.x), act_f64<ACT>(x.y));
+    if constexpr (sizeof(T) == 4) return act_f32<ACT>(x);
     else return act_bf16<ACT>(x);
 }
 

@@ -1,0 +1,62 @@
+"""Reproduces the polynomial coefficients hard-coded in fewbit_math.cuh.
+
+Run by hand (needs numpy and mpmath); prints the constants.  Not used at
+build or run time.
+
+1. GELU for bfloat16 storage.
+   x Phi(x) = max(x,0) - t Phi(-t), t = |x|, and
+   t Phi(-t) = t exp(-t^2/2) G(w),  w = 1/(1 + p t),  G(w) = p w (c0 + c1 w + c2 w^2 + c3 w^3).
+   Fit of (1 - w) (c0 + ... + c3 w^3) to t Phi(-t) exp(t^2/2) on t in (0, 14.5]
+   (note (1 - w) = p t w), relative error minimised by iteratively reweighted
+   least squares.  The kernel needs ~2^-10 relative accuracy.
+
+2. exp for binary32 storage.
+   e^r = 1 + r + r^2 Q(r) on |r| <= ln(2)/2, Q of degree 4, relative error of
+   e^r minimised the same way on Chebyshev nodes.
+"""
+import mpmath as mp
+import numpy as np
+
+mp.mp.dps = 40
+
+
+def minimax_lstsq(A, target, weight_of_error, iters=60):
+    w = np.ones(len(target))
+    for _ in range(iters):
+        c, *_ = np.linalg.lstsq(A * w[:, None], target * w, rcond=None)
+        err = weight_of_error(A @ c - target)
+        w = w * (1 + 4 * np.abs(err) / np.abs(err).max())
+        w /= w.mean()
+    return c, np.abs(err).max()
+
+
+def fit_gelu_bf16(p=0.30, terms=4):
+    ts = np.concatenate([np.linspace(1e-4, 1, 400), np.linspace(1, 14.5, 1200)])
+    tq = np.array([float(mp.mpf(t) * mp.ncdf(-mp.mpf(t)) * mp.exp(mp.mpf(t) ** 2 / 2)) for t in ts])
+    w = 1 / (1 + p * ts)
+    A = np.stack([(1 - w) * w ** i for i in range(terms)], 1)
+    c, err = minimax_lstsq(A / tq[:, None], np.ones_like(tq), lambda e: e)
+    return p * c, err          # coefficients of G(w) / w
+
+
+def fit_exp_f32(deg_q=4):
+    half = float(mp.log(2) / 2) * 1.0005
+    k = np.arange(400)
+    r = half * np.cos(np.pi * (k + 0.5) / 400)
+    target = np.array([float((mp.exp(mp.mpf(x)) - 1 - mp.mpf(x)) / mp.mpf(x) ** 2) for x in r])
+    A = np.stack([r ** i for i in range(deg_q + 1)], 1)
+    return minimax_lstsq(A, target, lambda e: e * r ** 2 / np.exp(r))
+
+
+if __name__ == "__main__":
+    c, err = fit_gelu_bf16()
+    print("GELU bf16: p = 0.30, G(w)/w coefficients (c0..c3):", [float(np.float32(v)) for v in c],
+          "max relative error %.3e" % err)
+    q, err = fit_exp_f32()
+    print("exp f32: Q coefficients (r^0..r^4):", [float(np.float32(v)) for v in q],
+          "max relative error of e^r %.3e (%.3f binary32 ulp)" % (err, err / 2 ** -24))
+    # Cody-Waite split of ln 2: the high part keeps 15 significant bits, so n * hi is exact for |n| < 512
+    ln2 = mp.log(2)
+    bits = np.array([float(ln2)], dtype=np.float32).view(np.uint32) & np.uint32(0xfffffe00)
+    hi = float(bits.view(np.float32)[0])
+    print("ln 2 split: hi = %.15g, lo = %.15g" % (hi, float(ln2 - mp.mpf(hi))))
