@@ -134,6 +134,12 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  * bytes is written.  n == 0 returns FEWBIT_OK without a launch.
  * Errors: FEWBIT_ERR_INVALID_ARG (NULL table or buffer, bad dtype),
  * FEWBIT_ERR_ALIGNMENT, FEWBIT_ERR_CUDA (launch failed).
+ * The interval search has several equivalent kernel variants (binary search,
+ * two-at-a-time bfloat16 search, shared-memory code table) chosen from bits,
+ * dtype and n; all give identical codes.  Two environment variables exist for
+ * testing and tuning only: FEWBIT_FWD_TABLE = always | never | auto (use of
+ * the code-table variant, default auto) and FEWBIT_FWD_ITERS = <k> (warp-blocks
+ * per warp).
  */
 FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y,
                                     uint32_t *packed, size_t n, fewbit_dtype dtype, void *stream);

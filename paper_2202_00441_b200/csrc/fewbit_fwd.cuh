@@ -302,6 +302,7 @@ constexpr size_t fwd_smem_bytes() {
 }
 
 int device_sm_count(cudaError_t *err);   // of the current device, cached
+constexpr size_t kLutMinIters = 8;      // below this many warp-blocks per warp the table does not pay for its expansion
 const char *fwd_iters_override();        // tuning aid: environment FEWBIT_FWD_ITERS
 
 template <int ACT, int BITS, typename T, bool LUT>
@@ -319,13 +320,17 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     constexpr size_t warps_per_cta = kFwdThreads / 32;
     const size_t warp_blocks = n / kWarpElems + ((n % kWarpElems) ? 1 : 0);
     // Iterations per warp.  Without a table: short CTAs, ~6 waves over the resident slots (the
-    // block scheduler evens out SMs that run slow), at most 8.  With a table the expansion has to
-    // be amortised: ~2 waves, at most 32.
-    constexpr size_t kMaxIters = LUT ? 32 : 8;
-    constexpr size_t kWaves = LUT ? 2 : 6;
+    // block scheduler evens out SMs that run slow), at most 8.  With a table its expansion has to
+    // be amortised: exactly one wave, every CTA resident from the start (the caller only picks
+    // the table variant when that gives each warp at least kLutMinIters iterations).
     const size_t slots = static_cast<size_t>(sms) * kFwdCtasPerSm;
-    size_t iters = warp_blocks / (warps_per_cta * slots * kWaves);
-    iters = iters < 1 ? 1 : (iters > kMaxIters ? kMaxIters : iters);
+    size_t iters;
+    if constexpr (LUT) {
+        iters = (warp_blocks + warps_per_cta * slots - 1) / (warps_per_cta * slots);
+    } else {
+        iters = warp_blocks / (warps_per_cta * slots * 6);
+        iters = iters < 1 ? 1 : (iters > 8 ? 8 : iters);
+    }
     if (const char *dbg = fwd_iters_override()) iters = static_cast<size_t>(atoi(dbg));
     const size_t per_cta = warps_per_cta * iters;
     const unsigned grid = static_cast<unsigned>((warp_blocks + per_cta - 1) / per_cta);

@@ -140,7 +140,16 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
     for (int m = 0; m < kMaxLevels; ++m) { prm.tb.s[m] = table->s[m]; prm.sb2[m] = table->s_bf16x2[m]; }
     const bool bf16 = dtype == FEWBIT_BF16;
     prm.runs = bf16 ? table->runs_bf16 : table->runs_f32;
-    const bool use_lut = prm.runs.count != 0;
+    // the shared-memory code table pays off only when every warp of a one-wave grid gets enough work
+    cudaError_t sm_err = cudaSuccess;
+    const size_t slots = static_cast<size_t>(device_sm_count(&sm_err)) * kFwdCtasPerSm;
+    if (sm_err != cudaSuccess) { t_last_cuda_error = static_cast<int>(sm_err); return FEWBIT_ERR_CUDA; }
+    const size_t warps_per_cta = static_cast<size_t>(bf16 ? FwdThreads<__nv_bfloat16>::value : FwdThreads<float>::value) / 32;
+    bool use_lut = prm.runs.count != 0 && n / kWarpElems >= kLutMinIters * warps_per_cta * slots;
+    if (const char *force = getenv("FEWBIT_FWD_TABLE")) {               // testing aid, see fewbit.h
+        if (force[0] == 'a') use_lut = prm.runs.count != 0;               // "always"
+        else if (force[0] == 'n') use_lut = false;                        // "never"
+    }
     const cudaError_t err = fwd_launchers(table->act).fn[table->bits - 1][bf16][use_lut](
         prm, x, y, packed, n, static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) { t_last_cuda_error = static_cast<int>(err); return FEWBIT_ERR_CUDA; }

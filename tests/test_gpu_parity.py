@@ -6,6 +6,7 @@ dtype of the exactly rounded binary64 value.  Both sides use the SAME table
 (read back from the library with fewbit_table_get), so the comparison isolates
 the hot path; the solver is compared with the oracle's DP in the CPU tests.
 """
+import os
 from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
@@ -191,9 +192,23 @@ def test_config5_sweep_large_sampled(n, dtype):
 # --------------------------------------------------------------------------
 # edge cases
 # --------------------------------------------------------------------------
+@pytest.fixture(params=["auto", "always", "never"])
+def table_mode(request):
+    """Runs a test under each bucketize variant: size-based choice, shared-memory
+    code table forced on (where the table has one), forced off."""
+    old = os.environ.get("FEWBIT_FWD_TABLE")
+    os.environ["FEWBIT_FWD_TABLE"] = request.param
+    yield request.param
+    if old is None:
+        os.environ.pop("FEWBIT_FWD_TABLE", None)
+    else:
+        os.environ["FEWBIT_FWD_TABLE"] = old
+
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("bits", [1, 2, 3, 4])
-def test_ragged_sizes(dtype, bits):
+def test_ragged_sizes(dtype, bits, table_mode):
     gen = torch.Generator(device=DEV).manual_seed(11)
     for n in [1, 7, 31, 32, 33, 255, 256, 257, 1023, 1024, 1025, 2047, 2048 + 33, 5 * 1024 + 1000, 9999]:
         x = (torch.randn(n, generator=gen, device=DEV) * 2).to(TORCH_DT[dtype])
@@ -213,7 +228,7 @@ def test_empty_input_is_a_no_op():
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
-def test_in_place_aliasing(dtype):
+def test_in_place_aliasing(dtype, table_mode):
     gen = torch.Generator(device=DEV).manual_seed(5)
     n = 70001
     x = torch.randn(n, generator=gen, device=DEV).to(TORCH_DT[dtype])
@@ -224,7 +239,7 @@ def test_in_place_aliasing(dtype):
 
 
 @pytest.mark.parametrize("act", wl.ACTIVATIONS)
-def test_every_bf16_pattern(act):
+def test_every_bf16_pattern(act, table_mode):
     """All 65 536 bfloat16 inputs: codes for every pattern (NaN and infinities
     included), y for every finite input."""
     h = torch.arange(65536, dtype=torch.int32).to(torch.int16).view(torch.bfloat16).to(DEV)
@@ -235,7 +250,7 @@ def test_every_bf16_pattern(act):
 
 
 @pytest.mark.parametrize("act", wl.ACTIVATIONS)
-def test_f32_values_around_every_boundary_and_in_the_tails(act):
+def test_f32_values_around_every_boundary_and_in_the_tails(act, table_mode):
     pieces = []
     for bits in (1, 2, 3, 4):
         s, _ = table(act, bits).arrays()
@@ -267,7 +282,7 @@ def test_gradient_specials_are_bit_exact():
             compare_full("gelu", bits, xs, g, y, p, gi, f"grad specials {dtype}")
 
 
-def test_injected_table_with_equal_boundaries():
+def test_injected_table_with_equal_boundaries(table_mode):
     s = np.array([-1.0, 0.0, 0.0, 0.0, 0.5, 0.5, 3.0], dtype=np.float32)
     lev = np.linspace(-1, 1, 8).astype(np.float32)
     t = fb.fewbit_table_from_arrays("elu", 3, s, lev)
@@ -280,6 +295,29 @@ def test_injected_table_with_equal_boundaries():
     gi_ref = oracle.bwd(3, lev, p_ref, np_bits(g))
     assert np.array_equal(np_bits(p).view(np.uint32), p_ref)
     assert np.array_equal(np_bits(gi), gi_ref)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_boundaries_closer_than_a_table_cell(dtype, table_mode):
+    """Boundaries a few binary32 ulps apart land in one cell of the binary32 code table (the warp
+    must fall back to the search there) and round to one bfloat16 (the packed search must still
+    count them separately)."""
+    base = np.float32(0.7431)
+    s = np.array([-1.0, base, np.nextafter(base, np.float32(1)), np.nextafter(np.nextafter(base, np.float32(1)), np.float32(1)),
+                  1.5, 1.5, 2.0], dtype=np.float32)
+    lev = np.arange(8, dtype=np.float32)
+    t = fb.fewbit_table_from_arrays("silu", 3, s, lev)
+    near = np.concatenate([np.nextafter(s, np.float32(-9)), s, np.nextafter(s, np.float32(9))])
+    x_np = np.concatenate([near, np.linspace(-3, 3, 50001).astype(np.float32), np.array([np.inf, -np.inf, np.nan], np.float32)])
+    x = torch.from_numpy(x_np).to(DEV).to(TORCH_DT[dtype])
+    g = torch.ones_like(x)
+    y, p = fb.fewbit_fwd(t, x)
+    gi = fb.fewbit_bwd(t, p, g)
+    torch.cuda.synchronize()
+    _, p_ref = oracle.fwd("silu", 3, s, np_bits(x))
+    gi_ref = oracle.bwd(3, lev, p_ref, np_bits(g))
+    assert np.array_equal(np_bits(p).view(np.uint32), p_ref)
+    assert np.array_equal(np_bits(gi).view(gi_ref.dtype), gi_ref)
 
 
 def test_misaligned_device_buffers_are_rejected():
