@@ -70,7 +70,8 @@ typedef enum fewbit_status {
     FEWBIT_ERR_UNSUPPORTED = 2,   /* valid request this build cannot serve                      */
     FEWBIT_ERR_ALIGNMENT = 3,     /* a buffer breaks the alignment rule of the call             */
     FEWBIT_ERR_CUDA = 4,          /* a CUDA call failed; see fewbit_last_cuda_error()           */
-    FEWBIT_ERR_ALLOC = 5          /* host allocation failed / workspace too small               */
+    FEWBIT_ERR_ALLOC = 5,         /* host allocation failed / workspace too small               */
+    FEWBIT_ERR_TOO_LARGE = 6      /* n exceeds the fixed capacity of an allocation-free call    */
 } fewbit_status;
 
 /* ------------------------------------------------------------------------- */
@@ -188,6 +189,42 @@ FEWBIT_API fewbit_status fewbit_bwd_host(const fewbit_table *table, const uint32
                                          const void *grad_out_host, void *grad_in_host, size_t n,
                                          fewbit_dtype dtype, void *workspace,
                                          size_t workspace_bytes);
+
+/*
+ * Forward half on HOST buffers WITHOUT any device allocation -- not even one
+ * made by the caller.  (The paper has no counterpart: this is a packaging
+ * variant of fewbit_fwd_host, same kernel, same results.)
+ *
+ * Who needs it: code that must not, or cannot, call cudaMalloc at the point
+ * where it wants the forward pass -- a plug-in running inside a host
+ * application whose memory pool already owns the whole device, a process held
+ * to a fixed device-memory budget, or a latency-sensitive loop that cannot
+ * afford the device-wide synchronisation an allocation may imply.  For them
+ * the staging area that fewbit_fwd_host expects as `workspace` is a fixed
+ * array inside the library image: FEWBIT_STATIC_MAX_ELEMS elements of room
+ * (about 2.1 MiB of device memory), held by every GPU on which the library is
+ * loaded until the process exits.
+ *
+ * x_host, y_host, packed_host: HOST buffers as in fewbit_fwd_host.  `stream`:
+ * the copies and the kernel are enqueued on it and it is synchronised before
+ * the call returns.  n > fewbit_static_max_elements() is rejected with
+ * FEWBIT_ERR_TOO_LARGE (split the tensor on a multiple of 1024 elements and
+ * call once per piece, or use fewbit_fwd_host).  The call makes no
+ * cudaMalloc / cudaFree and creates no stream or event.
+ *
+ * The first call on each device looks up the device address of the array
+ * (cudaGetSymbolAddress, with that device current); make that first call
+ * outside of any stream capture.  All calls on a device share the one array:
+ * it still holds the previous call's data (harmless -- every byte that is
+ * read is written first, so nothing needs clearing), and two calls whose GPU
+ * work overlaps in time, from different threads or streams, race on it.
+ * Serialise them.
+ */
+#define FEWBIT_STATIC_MAX_ELEMS 262144
+FEWBIT_API size_t fewbit_static_max_elements(void);
+FEWBIT_API fewbit_status fewbit_fwd_host_static(const fewbit_table *table, const void *x_host,
+                                                void *y_host, uint32_t *packed_host, size_t n,
+                                                fewbit_dtype dtype, void *stream);
 
 /* ------------------------------------------------------------------------- */
 /* Diagnostics                                                                */

@@ -63,6 +63,10 @@ def load_library():
     lib.fewbit_fwd_host.argtypes = [vp, vp, vp, vp, sz, ci, vp, sz]
     lib.fewbit_bwd_host.restype = ci
     lib.fewbit_bwd_host.argtypes = [vp, vp, vp, vp, sz, ci, vp, sz]
+    lib.fewbit_static_max_elements.restype = sz
+    lib.fewbit_static_max_elements.argtypes = []
+    lib.fewbit_fwd_host_static.restype = ci
+    lib.fewbit_fwd_host_static.argtypes = [vp, vp, vp, vp, sz, ci, vp]
     lib.fewbit_status_string.restype = ctypes.c_char_p
     lib.fewbit_status_string.argtypes = [ci]
     lib.fewbit_last_cuda_error.restype = ci
@@ -240,3 +244,26 @@ def fewbit_bwd_host(table: Table, packed: torch.Tensor, grad_out: torch.Tensor, 
                                    _DTYPES[grad_out.dtype], workspace.data_ptr(),
                                    workspace.numel() * workspace.element_size()), "fewbit_bwd_host")
     return grad_in
+
+
+def fewbit_static_max_elements() -> int:
+    return int(load_library().fewbit_static_max_elements())
+
+
+def fewbit_fwd_host_static(table: Table, x: torch.Tensor, y: torch.Tensor, packed: torch.Tensor,
+                           stream: Optional[torch.cuda.Stream] = None, device=None):
+    """Forward half on host tensors with no device allocation by anyone: the
+    device staging area is a fixed array inside the library (at most
+    ``fewbit_static_max_elements()`` elements per call).  For callers that
+    cannot call cudaMalloc where they need the forward pass.  Blocks until the
+    results are in ``y`` and ``packed``; calls must not overlap on one GPU."""
+    lib = load_library()
+    _host_tensor(x, "x"), _host_tensor(y, "y"), _host_tensor(packed, "packed")
+    n = x.numel()
+    if y.dtype != x.dtype or y.numel() != n or packed.numel() * packed.element_size() < fewbit_packed_bytes(n, table.bits):
+        raise ValueError("y / packed do not match x")
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(device):
+        _check(lib.fewbit_fwd_host_static(table.handle, x.data_ptr(), y.data_ptr(), packed.data_ptr(), n,
+                                          _DTYPES[x.dtype], _stream_ptr(stream, device)), "fewbit_fwd_host_static")
+    return y, packed

@@ -307,6 +307,7 @@ const char *fewbit_status_string(fewbit_status status) {
     case FEWBIT_ERR_ALIGNMENT: return "buffer alignment";
     case FEWBIT_ERR_CUDA: return "CUDA error";
     case FEWBIT_ERR_ALLOC: return "allocation failed or workspace too small";
+    case FEWBIT_ERR_TOO_LARGE: return "more elements than the fixed staging area of the allocation-free call holds";
     }
     return "unknown status";
 }
