@@ -374,7 +374,12 @@ def run_ours(args, case: wl.Case, act: str):
 
 # DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum of one launch / n) read from the
 # ncu captures summarised under profiles/; None until a capture exists for that kernel.
-NCU_TRAFFIC_BYTES_PER_ELEM = {}
+NCU_TRAFFIC_BYTES_PER_ELEM = {
+    # profiles/fwd_kernel_gelu_k4_bf16_2p27.md and profiles/bwd_kernel_k4_bf16_2p27.md (2^27 elements;
+    # scaled per element: a lower bound for the full launch, the L2 keeps ~55 MB of dirty lines either way)
+    ("bf16", "fwd_k4"): 4.078,
+    ("bf16", "bwd_k4"): 4.089,
+}
 
 
 def dataclass_replace_seed(case: wl.Case, seed: int) -> wl.Case:
