@@ -19,6 +19,7 @@ SOURCES += [("fewbit_fwd_inst.cu", f"fewbit_fwd_act{a}", [f"-DFEWBIT_ACT_ID={a}"
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC,-fvisibility=hidden,-O2", "-I", INCLUDE, "-I", CSRC,
+    *os.environ.get("FEWBIT_EXTRA_NVCC_FLAGS", "").split(),
 ]
 
 

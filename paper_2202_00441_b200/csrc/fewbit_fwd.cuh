@@ -63,6 +63,35 @@ __device__ __forceinline__ uint32_t cell(const Raw<__nv_bfloat16> &r, int e) {
     return (e & 1) ? (r.v[e >> 1] >> 16) : (r.v[e >> 1] & 0xffffu);
 }
 
+// ---------------------------------------------------------------------------
+// asynchronous prefetch ring (variants without a code table): every lane copies
+// its own lane-chunks of the next kStages warp-blocks global -> shared with
+// cp.async and reads the same bytes back just before use.  No lane reads what
+// another lane copied, so no barrier is involved; cp.async.wait_group is a
+// blocking instruction, not a spin loop.
+// ---------------------------------------------------------------------------
+#ifndef FEWBIT_ASYNC_STAGES
+#define FEWBIT_ASYNC_STAGES 2
+#endif
+
+__device__ __forceinline__ void cp_async_chunk(uint32_t saddr, const __nv_bfloat16 *g) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(saddr), "l"(g) : "memory");
+}
+__device__ __forceinline__ void cp_async_chunk(uint32_t saddr, const float *g) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(saddr), "l"(g) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(saddr + 16), "l"(g + 4) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
+
+__device__ __forceinline__ void load_raw_shared(uint32_t saddr, Raw<__nv_bfloat16> &r) {
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]) : "r"(saddr) : "memory");
+}
+__device__ __forceinline__ void load_raw_shared(uint32_t saddr, Raw<float> &r) {
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "r"(saddr) : "memory");
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7]) : "r"(saddr + 16) : "memory");
+}
+
 struct FwdSmem {
     uint32_t runs[kMaxRuns + 1];     // start | value << 24, plus a sentinel run starting one past the last cell
     uint32_t work[kMaxRuns + 1];     // [0] = count, then 16-cell groups that straddle a run boundary
@@ -167,7 +196,7 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
 // bfloat16: how many of the four element pairs of a lane-chunk use the look-up table when the
 // kernel has one (the rest use the packed search)
 #ifndef FEWBIT_LUT_PAIRS_K3
-#define FEWBIT_LUT_PAIRS_K3 4
+#define FEWBIT_LUT_PAIRS_K3 0
 #endif
 #ifndef FEWBIT_LUT_PAIRS_K4
 #define FEWBIT_LUT_PAIRS_K4 4
@@ -192,11 +221,30 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     const size_t cta_end = cta_begin + warps * iters;
     const size_t full = all_full < cta_end ? all_full : cta_end;                 // this CTA's warp-blocks are [cta_begin, full)
 
-    // Software pipeline: as soon as a tile of the current warp-block has been consumed, the same
-    // registers are reloaded with that tile of the warp's next warp-block, so four loads per lane
-    // stay in flight while the warp computes.
+    constexpr int kStages = LUT ? 0 : FEWBIT_ASYNC_STAGES;          // 0: prefetch into registers
+    constexpr uint32_t kChunkBytes = kLaneElems * sizeof(T);
+    constexpr uint32_t kStageBytes = kTilesPerWarp * 32 * kChunkBytes;          // one warp-block
+    [[maybe_unused]] uint32_t ring = 0, stage = 0;                  // this lane's slot base in the ring; stage in use
+    // Software pipeline.  Without a code table: the cp.async ring above, kStages warp-blocks ahead.
+    // With one (shared memory is taken): as soon as a tile of the current warp-block has been
+    // consumed, the same registers are reloaded with that tile of the warp's next warp-block, so
+    // four loads per lane stay in flight while the warp computes.
     Raw<T> cur[kTilesPerWarp];
-    if (warp0 < full) {
+    if constexpr (kStages > 0) {
+        ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw)) + (threadIdx.x >> 5) * (kStages * kStageBytes) +
+               lane * kChunkBytes;
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) {
+            const size_t wbs = warp0 + s * warps;
+            if (wbs < full) {
+                const T *px = x + wbs * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
+#pragma unroll
+                for (int t = 0; t < kTilesPerWarp; ++t)
+                    cp_async_chunk(ring + s * kStageBytes + t * (32 * kChunkBytes), px + t * kTileElems);
+            }
+            cp_async_commit();
+        }
+    } else if (warp0 < full) {
         const T *px = x + warp0 * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
 #pragma unroll
         for (int t = 0; t < kTilesPerWarp; ++t) load_raw(px + t * kTileElems, cur[t]);
@@ -212,8 +260,10 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         const T *px_next = x + base + warps * kWarpElems;
         const bool more = wb + warps < full;
         uint32_t grp[4];
+        if constexpr (kStages > 0) cp_async_wait<(kStages > 0 ? kStages - 1 : 0)>();   // the oldest stage has landed
 #pragma unroll
         for (int t = 0; t < kTilesPerWarp; ++t) {
+            if constexpr (kStages > 0) load_raw_shared(ring + stage * kStageBytes + t * (32 * kChunkBytes), cur[t]);
             float o[8];
             uint32_t g = 0;
             [[maybe_unused]] uint32_t dense = 0;
@@ -261,7 +311,20 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
             }
             grp[t] = g;
             store8(py + t * kTileElems, o);
-            if (more) load_raw(px_next + t * kTileElems, cur[t]);
+            if constexpr (kStages == 0) {
+                if (more) load_raw(px_next + t * kTileElems, cur[t]);
+            }
+        }
+        if constexpr (kStages > 0) {                               // refill the stage just consumed
+            const size_t wbn = wb + kStages * warps;
+            if (wbn < full) {
+                const T *px = x + wbn * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
+#pragma unroll
+                for (int t = 0; t < kTilesPerWarp; ++t)
+                    cp_async_chunk(ring + stage * kStageBytes + t * (32 * kChunkBytes), px + t * kTileElems);
+            }
+            cp_async_commit();
+            stage = (stage + 1 == kStages) ? 0 : stage + 1;
         }
         quad_transpose(grp, lane);
         uint32_t w[BITS];
@@ -298,7 +361,8 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
 
 template <typename T, bool LUT>
 constexpr size_t fwd_smem_bytes() {
-    return LUT ? (sizeof(T) == 2 ? (1u << kCellBitsBf16) : (1u << kCellBitsF32)) + sizeof(FwdSmem) : 0;
+    return LUT ? (sizeof(T) == 2 ? (1u << kCellBitsBf16) : (1u << kCellBitsF32)) + sizeof(FwdSmem)
+               : static_cast<size_t>(FEWBIT_ASYNC_STAGES) * (FwdThreads<T>::value / 32) * kWarpElems * sizeof(T);
 }
 
 int device_sm_count(cudaError_t *err);   // of the current device, cached
@@ -319,17 +383,18 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     constexpr int kFwdThreads = FwdThreads<T>::value;
     constexpr size_t warps_per_cta = kFwdThreads / 32;
     const size_t warp_blocks = n / kWarpElems + ((n % kWarpElems) ? 1 : 0);
-    // Iterations per warp.  Without a table: short CTAs, ~6 waves over the resident slots (the
-    // block scheduler evens out SMs that run slow), at most 8.  With a table its expansion has to
-    // be amortised: exactly one wave, every CTA resident from the start (the caller only picks
-    // the table variant when that gives each warp at least kLutMinIters iterations).
+    // Iterations per warp.  Without a table: short CTAs, ~8 waves over the resident slots (the
+    // block scheduler evens out SMs that run slow; the prefetch ring hides the pipeline fill), at
+    // most 4.  With a table its expansion has to be amortised: exactly one wave, every CTA resident
+    // from the start (the caller only picks the table variant when that gives each warp at least
+    // kLutMinIters iterations).
     const size_t slots = static_cast<size_t>(sms) * kFwdCtasPerSm;
     size_t iters;
     if constexpr (LUT) {
         iters = (warp_blocks + warps_per_cta * slots - 1) / (warps_per_cta * slots);
     } else {
-        iters = warp_blocks / (warps_per_cta * slots * 6);
-        iters = iters < 1 ? 1 : (iters > 8 ? 8 : iters);
+        iters = warp_blocks / (warps_per_cta * slots * 8);
+        iters = iters < 1 ? 1 : (iters > 4 ? 4 : iters);
     }
     if (const char *dbg = fwd_iters_override()) iters = static_cast<size_t>(atoi(dbg));
     const size_t per_cta = warps_per_cta * iters;
