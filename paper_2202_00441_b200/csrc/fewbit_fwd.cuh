@@ -31,6 +31,7 @@
 // LUT = false: no table (bfloat16: packed search; binary32: search).
 #pragma once
 
+#include <atomic>
 #include <cstdlib>
 
 #include "fewbit_device.cuh"
@@ -376,9 +377,17 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     if (err != cudaSuccess) return err;
     constexpr size_t smem = fwd_smem_bytes<T, LUT>();
     auto kernel = fwd_kernel<ACT, BITS, T, LUT>;
-    if constexpr (smem > 48 * 1024) {
-        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if constexpr (smem > 48 * 1024) {           // opt in to the large dynamic shared memory once per device
+        static std::atomic<uint64_t> opted_in{0};
+        int dev = 0;
+        err = cudaGetDevice(&dev);
         if (err != cudaSuccess) return err;
+        const uint64_t bit = 1ull << (dev & 63);
+        if (!(opted_in.load(std::memory_order_relaxed) & bit)) {
+            err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+            if (err != cudaSuccess) return err;
+            opted_in.fetch_or(bit, std::memory_order_relaxed);
+        }
     }
     constexpr int kFwdThreads = FwdThreads<T>::value;
     constexpr size_t warps_per_cta = kFwdThreads / 32;

@@ -188,9 +188,51 @@ __device__ __forceinline__ float2 neg_logistic_tail_scaled_f32(float2 x) {
     return fma2(res, rn, qn);                                                // -(q0 + res / Dh)
 }
 
+// GELU for binary32 storage, in binary64 with purpose-built pieces (the binary32 result then
+// carries a single rounding):  x Phi(x) = max(x,0) - t Phi(-t),  t = |x|,
+// Phi(-t) = e^{-t^2/2} w P(z),  w = 1/(1 + 0.3 t),  z = A w + B in [-1,1], P of degree 9 fitted to
+// Phi(-t) e^{t^2/2} / w on t in [0,15] (relative error 3.5e-9 = 0.06 binary32 ulp; fit_coefficients.py).
+// t^2 is exact in binary64 for a binary32 t.  Beyond t = 15 the subtracted term is 0 in binary32.
+__device__ __forceinline__ float gelu_f32_via_f64(float xf) {
+    const double x = static_cast<double>(xf);
+    const double t = fmin(fabs(x), 15.0);
+    // e^a, a = -t^2/2 in [-112.5, 0]: n = round(a log2 e), r = a - n ln 2 (two pieces), degree-8 Taylor
+    const double a = -0.5 * (t * t);
+    const double tn = fma(a, 1.4426950408889634, 6755399441055744.0);            // 1.5 * 2^52 + n
+    const double n = tn - 6755399441055744.0;
+    double r = fma(n, -0.693147180369123816490, a);
+    r = fma(n, -1.90821492927058770002e-10, r);
+    double e = fma(r, 2.48015873015873015873e-05, 1.98412698412698412698e-04);
+    e = fma(e, r, 1.38888888888888888889e-03);
+    e = fma(e, r, 8.33333333333333333333e-03);
+    e = fma(e, r, 4.16666666666666666667e-02);
+    e = fma(e, r, 1.66666666666666666667e-01);
+    e = fma(e, r, 0.5);
+    e = fma(e, r, 1.0);
+    e = fma(e, r, 1.0);
+    e *= __hiloint2double((__double2loint(tn) + 1023) << 20, 0);                 // * 2^n
+    // w = 1 / (1 + 0.3 t): hardware seed, one Newton step (2^-23 -> 2^-46)
+    const double d = fma(t, 0.3, 1.0);
+    double w = static_cast<double>(rcp_ftz(static_cast<float>(d)));
+    w = fma(w, fma(-d, w, 1.0), w);
+    const double z = fma(w, 2.4444444444444446, -1.4444444444444446);
+    double g = fma(z, -6.6198732346359193e-06, 2.1633418658465733e-06);
+    g = fma(g, z, 8.448490689851325e-05);
+    g = fma(g, z, -4.8574085770614277e-05);
+    g = fma(g, z, -0.0010375821171958151);
+    g = fma(g, z, -0.00027144998454187153);
+    g = fma(g, z, 0.015457929415072305);
+    g = fma(g, z, 0.068212812609166992);
+    g = fma(g, z, 0.16268319230647843);
+    g = fma(g, z, 0.25492364174848237);
+    return static_cast<float>(fmax(x, 0.0) - t * (e * (g * w)));
+}
+
 template <int ACT>
 __device__ __forceinline__ float2 act_f32(float2 x) {
-    if constexpr (ACT == FEWBIT_SILU) {
+    if constexpr (ACT == FEWBIT_GELU) {
+        return make_float2(gelu_f32_via_f64(x.x), gelu_f32_via_f64(x.y));
+    } else if constexpr (ACT == FEWBIT_SILU) {
         // x < 0: x q;  x >= 0: x - x q   with q = E / (1 + E)
         // below -131 the product is 0 in binary32; clamping there keeps |x| E from growing again
         // once E itself has been clamped
