@@ -42,7 +42,12 @@ namespace fewbit {
 // threads per CTA: binary32 keeps 32 registers of input in flight per thread, so it runs fewer,
 // fatter threads (register cap 80) than bfloat16 (cap 64)
 template <typename T> struct FwdThreads { static constexpr int value = sizeof(T) == 2 ? 512 : 384; };
+#ifndef FEWBIT_CTAS_NOLUT_BF16
+#define FEWBIT_CTAS_NOLUT_BF16 2
+#endif
 constexpr int kFwdCtasPerSm = 2;
+// resident CTAs per SM the kernel is compiled for (register cap = 65536 / threads / this)
+template <typename T, bool LUT> struct FwdCtas { static constexpr int value = (!LUT && sizeof(T) == 2) ? FEWBIT_CTAS_NOLUT_BF16 : kFwdCtasPerSm; };
 
 template <typename T> struct Raw;                 // the 8 elements of a lane-chunk as loaded
 template <> struct Raw<float> { float v[8]; };
@@ -205,7 +210,7 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
 template <int BITS> struct Bf16LutPairs { static constexpr int value = BITS == 4 ? FEWBIT_LUT_PAIRS_K4 : (BITS == 3 ? FEWBIT_LUT_PAIRS_K3 : 0); };
 
 template <int ACT, int BITS, typename T, bool LUT>
-__global__ void __launch_bounds__(FwdThreads<T>::value, kFwdCtasPerSm)
+__global__ void __launch_bounds__(FwdThreads<T>::value, FwdCtas<T, LUT>::value)
 fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters) {
     constexpr bool kIsBf16 = sizeof(T) == 2;
     constexpr int kFwdThreads = FwdThreads<T>::value;
@@ -397,7 +402,7 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     // most 4.  With a table its expansion has to be amortised: exactly one wave, every CTA resident
     // from the start (the caller only picks the table variant when that gives each warp at least
     // kLutMinIters iterations).
-    const size_t slots = static_cast<size_t>(sms) * kFwdCtasPerSm;
+    const size_t slots = static_cast<size_t>(sms) * FwdCtas<T, LUT>::value;
     size_t iters;
     if constexpr (LUT) {
         iters = (warp_blocks + warps_per_cta * slots - 1) / (warps_per_cta * slots);
