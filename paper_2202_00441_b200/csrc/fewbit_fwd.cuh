@@ -41,13 +41,26 @@ namespace fewbit {
 
 // threads per CTA: binary32 keeps 32 registers of input in flight per thread, so it runs fewer,
 // fatter threads (register cap 80) than bfloat16 (cap 64)
-template <typename T> struct FwdThreads { static constexpr int value = sizeof(T) == 2 ? 512 : 384; };
+#ifndef FEWBIT_LUT_THREADS_BF16
+#define FEWBIT_LUT_THREADS_BF16 512
+#endif
+#ifndef FEWBIT_LUT_CTAS_BF16
+#define FEWBIT_LUT_CTAS_BF16 2
+#endif
+#ifndef FEWBIT_LUT_STAGES_BF16
+#define FEWBIT_LUT_STAGES_BF16 1
+#endif
+template <typename T, bool LUT = false> struct FwdThreads {
+    static constexpr int value = sizeof(T) == 2 ? (LUT ? FEWBIT_LUT_THREADS_BF16 : 512) : 384;
+};
 #ifndef FEWBIT_CTAS_NOLUT_BF16
 #define FEWBIT_CTAS_NOLUT_BF16 2
 #endif
 constexpr int kFwdCtasPerSm = 2;
 // resident CTAs per SM the kernel is compiled for (register cap = 65536 / threads / this)
-template <typename T, bool LUT> struct FwdCtas { static constexpr int value = (!LUT && sizeof(T) == 2) ? FEWBIT_CTAS_NOLUT_BF16 : kFwdCtasPerSm; };
+template <typename T, bool LUT> struct FwdCtas {
+    static constexpr int value = sizeof(T) == 2 ? (LUT ? FEWBIT_LUT_CTAS_BF16 : FEWBIT_CTAS_NOLUT_BF16) : kFwdCtasPerSm;
+};
 
 template <typename T> struct Raw;                 // the 8 elements of a lane-chunk as loaded
 template <> struct Raw<float> { float v[8]; };
@@ -210,10 +223,10 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
 template <int BITS> struct Bf16LutPairs { static constexpr int value = BITS == 4 ? FEWBIT_LUT_PAIRS_K4 : (BITS == 3 ? FEWBIT_LUT_PAIRS_K3 : 0); };
 
 template <int ACT, int BITS, typename T, bool LUT>
-__global__ void __launch_bounds__(FwdThreads<T>::value, FwdCtas<T, LUT>::value)
+__global__ void __launch_bounds__(FwdThreads<T, LUT>::value, FwdCtas<T, LUT>::value)
 fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters) {
     constexpr bool kIsBf16 = sizeof(T) == 2;
-    constexpr int kFwdThreads = FwdThreads<T>::value;
+    constexpr int kFwdThreads = FwdThreads<T, LUT>::value;
     constexpr int kCells = kIsBf16 ? (1 << kCellBitsBf16) : (1 << kCellBitsF32);
     extern __shared__ __align__(16) uint8_t smem_raw[];
     uint8_t *lut = smem_raw;
@@ -227,7 +240,8 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     const size_t cta_end = cta_begin + warps * iters;
     const size_t full = all_full < cta_end ? all_full : cta_end;                 // this CTA's warp-blocks are [cta_begin, full)
 
-    constexpr int kStages = LUT ? 0 : FEWBIT_ASYNC_STAGES;          // 0: prefetch into registers
+    constexpr int kStages = LUT ? (kIsBf16 ? FEWBIT_LUT_STAGES_BF16 : 0) : FEWBIT_ASYNC_STAGES;   // 0: prefetch into registers
+    constexpr uint32_t kRingOffset = LUT ? (kCells + static_cast<uint32_t>(sizeof(FwdSmem)) + 127u) / 128u * 128u : 0u;
     constexpr uint32_t kChunkBytes = kLaneElems * sizeof(T);
     constexpr uint32_t kStageBytes = kTilesPerWarp * 32 * kChunkBytes;          // one warp-block
     [[maybe_unused]] uint32_t ring = 0, stage = 0;                  // this lane's slot base in the ring; stage in use
@@ -237,7 +251,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     // four loads per lane stay in flight while the warp computes.
     Raw<T> cur[kTilesPerWarp];
     if constexpr (kStages > 0) {
-        ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw)) + (threadIdx.x >> 5) * (kStages * kStageBytes) +
+        ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw)) + kRingOffset + (threadIdx.x >> 5) * (kStages * kStageBytes) +
                lane * kChunkBytes;
 #pragma unroll
         for (int s = 0; s < kStages; ++s) {
@@ -367,7 +381,8 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
 
 template <typename T, bool LUT>
 constexpr size_t fwd_smem_bytes() {
-    return LUT ? (sizeof(T) == 2 ? (1u << kCellBitsBf16) : (1u << kCellBitsF32)) + sizeof(FwdSmem)
+    return LUT ? ((sizeof(T) == 2 ? (1u << kCellBitsBf16) : (1u << kCellBitsF32)) + sizeof(FwdSmem) + 127u) / 128u * 128u +
+                     (sizeof(T) == 2 ? static_cast<size_t>(FEWBIT_LUT_STAGES_BF16) * (FwdThreads<T, true>::value / 32) * kWarpElems * sizeof(T) : 0)
                : static_cast<size_t>(FEWBIT_ASYNC_STAGES) * (FwdThreads<T>::value / 32) * kWarpElems * sizeof(T);
 }
 
@@ -394,7 +409,7 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
             opted_in.fetch_or(bit, std::memory_order_relaxed);
         }
     }
-    constexpr int kFwdThreads = FwdThreads<T>::value;
+    constexpr int kFwdThreads = FwdThreads<T, LUT>::value;
     constexpr size_t warps_per_cta = kFwdThreads / 32;
     const size_t warp_blocks = n / kWarpElems + ((n % kWarpElems) ? 1 : 0);
     // Iterations per warp.  Without a table: short CTAs, ~8 waves over the resident slots (the

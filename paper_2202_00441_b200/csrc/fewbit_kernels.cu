@@ -142,9 +142,9 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
     prm.runs = bf16 ? table->runs_bf16 : table->runs_f32;
     // the shared-memory code table pays off only when every warp of a one-wave grid gets enough work
     cudaError_t sm_err = cudaSuccess;
-    const size_t slots = static_cast<size_t>(device_sm_count(&sm_err)) * kFwdCtasPerSm;
+    const size_t slots = static_cast<size_t>(device_sm_count(&sm_err)) * (bf16 ? FwdCtas<__nv_bfloat16, true>::value : FwdCtas<float, true>::value);
     if (sm_err != cudaSuccess) { t_last_cuda_error = static_cast<int>(sm_err); return FEWBIT_ERR_CUDA; }
-    const size_t warps_per_cta = static_cast<size_t>(bf16 ? FwdThreads<__nv_bfloat16>::value : FwdThreads<float>::value) / 32;
+    const size_t warps_per_cta = static_cast<size_t>(bf16 ? FwdThreads<__nv_bfloat16, true>::value : FwdThreads<float, true>::value) / 32;
     bool use_lut = prm.runs.count != 0 && n / kWarpElems >= kLutMinIters * warps_per_cta * slots;
     if (const char *force = getenv("FEWBIT_FWD_TABLE")) {               // testing aid, see fewbit.h
         if (force[0] == 'a') use_lut = prm.runs.count != 0;               // "always"
