@@ -75,6 +75,10 @@ def _load():
             fn = getattr(lib, name)
             fn.restype = None
             fn.argtypes = [ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, sz]
+        for name in ("fbo_fwd_f32_fold", "fbo_fwd_bf16_fold"):
+            fn = getattr(lib, name)
+            fn.restype = None
+            fn.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, sz]
         for name in ("fbo_bwd_f32", "fbo_bwd_bf16"):
             fn = getattr(lib, name)
             fn.restype = None
@@ -213,11 +217,20 @@ def _check_tables(bits, s=None, lev=None):
     return s, lev
 
 
-def fwd(name, bits: int, s, x: np.ndarray):
+def dp_solve_folded(name, bits, B=8.0, n_cells=2048):
+    """Table for an even f' (caption of Fig. 3): 2^bits pieces on [0, B]; the
+    error over [-B, B] is twice the half-axis optimum."""
+    r = dp_solve(name, bits, 0.0, B, n_cells)
+    r["objective"] = 2.0 * r["objective"]
+    return r
+
+
+def fwd(name, bits: int, s, x: np.ndarray, fold: bool = False):
     """Forward half: returns (y, packed).
 
     ``x`` is float32, or uint16 holding bfloat16 bit patterns; ``y`` has the
-    same dtype.  ``s`` are the K-1 boundaries as binary32."""
+    same dtype.  ``s`` are the K-1 boundaries as binary32.  ``fold``: the code
+    is the position of |x| (table on [0, B] for an even f')."""
     s, _ = _check_tables(bits, s=s)
     if s.size == 0:
         s = np.zeros(1, dtype=np.float32)
@@ -227,9 +240,9 @@ def fwd(name, bits: int, s, x: np.ndarray):
     y = np.empty_like(x)
     lib = _load()
     if x.dtype == np.float32:
-        lib.fbo_fwd_f32(_act_id(name), int(bits), _ptr(s), _ptr(x), _ptr(y), _ptr(packed), n)
+        lib.fbo_fwd_f32_fold(_act_id(name), int(bits), int(bool(fold)), _ptr(s), _ptr(x), _ptr(y), _ptr(packed), n)
     elif x.dtype == np.uint16:
-        lib.fbo_fwd_bf16(_act_id(name), int(bits), _ptr(s), _ptr(x), _ptr(y), _ptr(packed), n)
+        lib.fbo_fwd_bf16_fold(_act_id(name), int(bits), int(bool(fold)), _ptr(s), _ptr(x), _ptr(y), _ptr(packed), n)
     else:
         raise TypeError("x must be float32 or uint16 (bfloat16 bits)")
     return y, packed

@@ -20,6 +20,9 @@
  *   fbo_fwd_*                 Listing 1 "forward": y = f(x); code = position
  *                             of x among the boundaries s (Eq. 2); only
  *                             log2(K) bits per element are kept (Sec. 2)
+ *   fbo_fwd_*_fold            the same with the position of |x| (caption of
+ *                             Fig. 3: for an even f' only the positive half-axis
+ *                             is quantised, the table lives on [0, B])
  *   fbo_bwd_*                 Listing 1 "backward": grad_in = grad_out * y[code]
  *
  * Every function here is pinned by tests/test_oracle_*.py against Table 1,
@@ -350,26 +353,41 @@ void fbo_unpack(int bits, const uint32_t *packed, uint8_t *codes, size_t n)
     for (size_t e = 0; e < n; ++e) codes[e] = (uint8_t)get_code(packed, e, bits);
 }
 
-void fbo_fwd_f32(int act, int bits, const float *s, const float *x, float *y,
-                 uint32_t *packed, size_t n)
+/* fold != 0: the table approximates an even f' on [0, B] and the code is the position of |x|
+ * (caption of Fig. 3).  y is unaffected. */
+void fbo_fwd_f32_fold(int act, int bits, int fold, const float *s, const float *x, float *y,
+                      uint32_t *packed, size_t n)
 {
     int nb = (1 << bits) - 1;
     memset(packed, 0, 4 * fbo_packed_words(n, bits));
     for (size_t e = 0; e < n; ++e) {
         y[e] = (float)fbo_act(act, (double)x[e]);
-        put_code(packed, e, bits, bucketize(s, nb, x[e]));
+        put_code(packed, e, bits, bucketize(s, nb, fold ? fabsf(x[e]) : x[e]));
     }
+}
+
+void fbo_fwd_bf16_fold(int act, int bits, int fold, const float *s, const uint16_t *x, uint16_t *y,
+                       uint32_t *packed, size_t n)
+{
+    int nb = (1 << bits) - 1;
+    memset(packed, 0, 4 * fbo_packed_words(n, bits));
+    for (size_t e = 0; e < n; ++e) {
+        float xf = bf16_to_f32(x[e]);
+        y[e] = fbo_f64_to_bf16(fbo_act(act, fbo_bf16_to_f64(x[e])));
+        put_code(packed, e, bits, bucketize(s, nb, fold ? fabsf(xf) : xf));
+    }
+}
+
+void fbo_fwd_f32(int act, int bits, const float *s, const float *x, float *y,
+                 uint32_t *packed, size_t n)
+{
+    fbo_fwd_f32_fold(act, bits, 0, s, x, y, packed, n);
 }
 
 void fbo_fwd_bf16(int act, int bits, const float *s, const uint16_t *x, uint16_t *y,
                   uint32_t *packed, size_t n)
 {
-    int nb = (1 << bits) - 1;
-    memset(packed, 0, 4 * fbo_packed_words(n, bits));
-    for (size_t e = 0; e < n; ++e) {
-        y[e] = fbo_f64_to_bf16(fbo_act(act, fbo_bf16_to_f64(x[e])));
-        put_code(packed, e, bits, bucketize(s, nb, bf16_to_f32(x[e])));
-    }
+    fbo_fwd_bf16_fold(act, bits, 0, s, x, y, packed, n);
 }
 
 /* ------------------------------------------------------------------------ */

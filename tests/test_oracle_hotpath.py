@@ -267,3 +267,27 @@ def test_backward_applies_the_piecewise_constant_function():
     np.testing.assert_array_equal(gi, q)
     # and q tracks f' with the error the table promises (mean square under N(0,1.5^2) is small)
     assert np.mean((gi - oracle.act_deriv("silu", x)) ** 2) < 0.02
+
+
+# --------------------------------------------------------------------------
+# even-derivative fold
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("bits", [1, 2, 4])
+def test_folded_bucketize_is_searchsorted_of_abs(bits):
+    r = oracle.dp_solve_folded("tanh", bits)
+    s, lev = r["s"].astype(np.float32), r["lev"].astype(np.float32)
+    x = np.concatenate([RNG.standard_normal(4000) * 2, s, -s, np.nextafter(s, np.float32(9)), -np.nextafter(s, np.float32(9)),
+                        [0.0, -0.0, np.inf, -np.inf, np.nan]]).astype(np.float32)
+    _, packed = oracle.fwd("tanh", bits, s, x, fold=True)
+    codes = oracle.unpack(packed, bits, x.size)
+    with np.errstate(invalid="ignore"):
+        ref = np.searchsorted(s, np.abs(x), side="left")
+    ref[np.isnan(x)] = 0
+    np.testing.assert_array_equal(codes, ref)
+    # the factor applied in the backward pass is an even function of x
+    gi = oracle.bwd(bits, lev, packed, np.ones_like(x))
+    _, packed_neg = oracle.fwd("tanh", bits, s, -x, fold=True)
+    np.testing.assert_array_equal(gi, oracle.bwd(bits, lev, packed_neg, np.ones_like(x)))
+    h, f = all_finite_bf16()
+    _, pb = oracle.fwd("tanh", bits, s, h, fold=True)
+    np.testing.assert_array_equal(oracle.unpack(pb, bits, h.size), np.searchsorted(s, np.abs(f), side="left"))

@@ -194,3 +194,30 @@ def test_config1_table_values():
     assert r["s"][3] == 0.0
     assert (r["s"].astype(np.float32).astype(np.float64) == r["s"]).all()
     assert (np.diff(r["lev"][1:-1]) > 0).all()
+
+
+# --------------------------------------------------------------------------
+# even-derivative fold (caption of Fig. 3)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["sigmoid", "tanh"])
+@pytest.mark.parametrize("bits", [1, 2, 3])
+def test_folded_table_is_worth_about_one_more_bit(name, bits):
+    """2^bits pieces on the half-axis are 2^(bits+1) symmetric pieces on the whole axis: the
+    error lies between the unfolded optimum with 2^(bits+1) pieces (nothing symmetric can beat
+    it) and the unfolded optimum with 2^bits pieces."""
+    folded = oracle.dp_solve_folded(name, bits, 8.0, 512)["objective"]
+    same_bits = oracle.dp_solve(name, bits, -8.0, 8.0, 1024)["objective"]
+    one_more = oracle.dp_solve(name, bits + 1, -8.0, 8.0, 1024)["objective"]
+    assert one_more - 1e-12 <= folded < same_bits
+    assert folded < 0.6 * same_bits
+
+
+@pytest.mark.parametrize("name", ["sigmoid", "tanh"])
+def test_folded_levels_are_means_over_the_half_axis_bins(name):
+    r = oracle.dp_solve_folded(name, 2, 8.0, 2048)
+    edges = np.concatenate([[0.0], r["s"], [8.0]])
+    assert (r["s"] > 0).all()
+    for m in range(4):
+        a, b = edges[m], edges[m + 1]
+        mean = (float(MP_F[name](mp.mpf(b))) - float(MP_F[name](mp.mpf(a)))) / (b - a)
+        assert r["lev"][m] == pytest.approx(mean, abs=1e-12)
