@@ -343,6 +343,7 @@ def run_ours(args, case: wl.Case, act: str):
         for name in ("c2", "c4", "c1"):
             if wl.CONFIGS[name].name != case.name:
                 also[name] = quick_config(fb, wl.CONFIGS[name], dev)
+        also["c4_folded"] = quick_config(fb, wl.C4, dev, folded=True)      # even-derivative fold: codes from |x|
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
@@ -411,7 +412,7 @@ def torch_unfused(case: wl.Case, act: str, x, g, reps: int = 5):
             "saved_bytes_per_elem": eb, "note": "stock torch forward + autograd backward, full input kept"}
 
 
-def quick_config(fb, case: wl.Case, dev, reps: int = 10):
+def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False):
     """Device-resident timing of another configuration.  L2-cold by rotation: enough independent
     buffer sets that their footprint exceeds 4x the 126 MB L2, a different set for every launch
     (a write-flush would leave the L2 full of dirty lines whose write-back is then charged to a
@@ -427,8 +428,10 @@ def quick_config(fb, case: wl.Case, dev, reps: int = 10):
     gis = [torch.empty_like(g0) for _ in range(sets)]
     out = {}
     for act in case.acts:
+        if folded and act not in ("sigmoid", "tanh"):
+            continue
         for b in case.bits:
-            t = fb.fewbit_table_create(act, b)
+            t = fb.fewbit_table_create_folded(act, b) if folded else fb.fewbit_table_create(act, b)
             ps = [torch.empty(fb.fewbit_packed_bytes(case.n, b) // 4, dtype=torch.int32, device=dev) for _ in range(sets)]
             f_ms, b_ms = [], []
             for i in range(reps + 3):

@@ -104,6 +104,26 @@ FEWBIT_API fewbit_status fewbit_table_create_ex(fewbit_act act, int bits, double
 FEWBIT_API fewbit_status fewbit_table_from_arrays(fewbit_act act, int bits, const float *s,
                                                   const float *lev, fewbit_table **out);
 
+/*
+ * Folded table for an activation whose derivative is even (caption of Fig. 3:
+ * "we can quantize only positive real axis", which is worth one more bit):
+ * 2^bits pieces on [0, B], found by the same dynamic programme on a grid of
+ * n_cells cells; the code of x is then #{ j : s[j] < |x| }.  Defined for
+ * FEWBIT_SIGMOID and FEWBIT_TANH, otherwise FEWBIT_ERR_UNSUPPORTED.  The
+ * objective reported by fewbit_table_get is the error over [-B, B] (twice the
+ * half-axis value).  fewbit_fwd / fewbit_bwd take such a table like any other.
+ * Suggested: B = 8, n_cells = 2048 (the grid step of the default tables).
+ */
+FEWBIT_API fewbit_status fewbit_table_create_folded(fewbit_act act, int bits, double B, int n_cells,
+                                                    fewbit_table **out);
+
+/* fewbit_table_from_arrays with the folded flag (folded != 0: s are boundaries of |x|). */
+FEWBIT_API fewbit_status fewbit_table_from_arrays_ex(fewbit_act act, int bits, const float *s,
+                                                     const float *lev, int folded, fewbit_table **out);
+
+/* 1 if the table is folded, else 0 (also for NULL). */
+FEWBIT_API int fewbit_table_is_folded(const fewbit_table *table);
+
 /* Frees a table; NULL is accepted. */
 FEWBIT_API void fewbit_table_destroy(fewbit_table *table);
 

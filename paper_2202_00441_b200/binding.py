@@ -47,6 +47,12 @@ def load_library():
     lib.fewbit_table_create_ex.argtypes = [ci, ci, ctypes.c_double, ctypes.c_double, ci, ctypes.POINTER(vp)]
     lib.fewbit_table_from_arrays.restype = ci
     lib.fewbit_table_from_arrays.argtypes = [ci, ci, vp, vp, ctypes.POINTER(vp)]
+    lib.fewbit_table_create_folded.restype = ci
+    lib.fewbit_table_create_folded.argtypes = [ci, ci, ctypes.c_double, ci, ctypes.POINTER(vp)]
+    lib.fewbit_table_from_arrays_ex.restype = ci
+    lib.fewbit_table_from_arrays_ex.argtypes = [ci, ci, vp, vp, ci, ctypes.POINTER(vp)]
+    lib.fewbit_table_is_folded.restype = ci
+    lib.fewbit_table_is_folded.argtypes = [vp]
     lib.fewbit_table_destroy.restype = None
     lib.fewbit_table_destroy.argtypes = [vp]
     lib.fewbit_table_get.restype = ci
@@ -97,6 +103,7 @@ class Table:
         _check(load_library().fewbit_table_get(self._h, ctypes.byref(act), ctypes.byref(bits), None, None,
                                                ctypes.byref(obj)), "fewbit_table_get")
         self.act, self.bits, self.objective = act.value, bits.value, obj.value
+        self.folded = bool(load_library().fewbit_table_is_folded(self._h))
 
     @property
     def handle(self):
@@ -130,7 +137,15 @@ def fewbit_table_create_ex(act, bits: int, A: float, B: float, n_cells: int) -> 
     return Table(out.value or 0)
 
 
-def fewbit_table_from_arrays(act, bits: int, s, lev) -> Table:
+def fewbit_table_create_folded(act, bits: int, B: float = 8.0, n_cells: int = 2048) -> Table:
+    """Folded table (even derivative: sigmoid, tanh): 2^bits pieces on [0, B], codes from |x|."""
+    out = ctypes.c_void_p()
+    _check(load_library().fewbit_table_create_folded(_act_id(act), int(bits), float(B), int(n_cells),
+                                                     ctypes.byref(out)), "fewbit_table_create_folded")
+    return Table(out.value or 0)
+
+
+def fewbit_table_from_arrays(act, bits: int, s, lev, folded: bool = False) -> Table:
     import numpy as np
 
     s = np.ascontiguousarray(s, dtype=np.float32)
@@ -141,8 +156,8 @@ def fewbit_table_from_arrays(act, bits: int, s, lev) -> Table:
     if s.size == 0:
         s = np.zeros(1, dtype=np.float32)
     out = ctypes.c_void_p()
-    _check(load_library().fewbit_table_from_arrays(_act_id(act), int(bits), s.ctypes.data, lev.ctypes.data,
-                                                   ctypes.byref(out)), "fewbit_table_from_arrays")
+    _check(load_library().fewbit_table_from_arrays_ex(_act_id(act), int(bits), s.ctypes.data, lev.ctypes.data,
+                                                      int(bool(folded)), ctypes.byref(out)), "fewbit_table_from_arrays")
     return Table(out.value or 0)
 
 

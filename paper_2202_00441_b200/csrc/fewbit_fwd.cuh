@@ -222,7 +222,9 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
 #endif
 template <int BITS> struct Bf16LutPairs { static constexpr int value = BITS == 4 ? FEWBIT_LUT_PAIRS_K4 : (BITS == 3 ? FEWBIT_LUT_PAIRS_K3 : 0); };
 
-template <int ACT, int BITS, typename T, bool LUT>
+// FOLD: the code is the position of |x| (even f', table on [0, B]); the code tables arrive already
+// built that way, the searches strip the sign first.
+template <int ACT, int BITS, typename T, bool LUT, bool FOLD>
 __global__ void __launch_bounds__(FwdThreads<T, LUT>::value, FwdCtas<T, LUT>::value)
 fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters) {
     constexpr bool kIsBf16 = sizeof(T) == 2;
@@ -298,18 +300,19 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
                     if (LUT && (e / 2) < Bf16LutPairs<BITS>::value) {              // resolved at compile time (unrolled)
                         pc[e / 2] = lut[cell(cur[t], e)] + (static_cast<uint32_t>(lut[cell(cur[t], e + 1)]) << 16);
                     } else {
-                        pc[e / 2] = bucketize_bf16x2<BITS>(prm.sb2, pair_bits(cur[t], e));
+                        pc[e / 2] = bucketize_bf16x2<BITS>(prm.sb2, FOLD ? (pair_bits(cur[t], e) & 0x7fff7fffu) : pair_bits(cur[t], e));
                     }
                 } else {
                     uint32_t c0, c1;
+                    const float k0 = FOLD ? fabsf(xv.x) : xv.x, k1 = FOLD ? fabsf(xv.y) : xv.y;   // what is searched for
                     if constexpr (!LUT) {
-                        c0 = bucketize<BITS>(prm.tb, xv.x);
-                        c1 = bucketize<BITS>(prm.tb, xv.y);
+                        c0 = bucketize<BITS>(prm.tb, k0);
+                        c1 = bucketize<BITS>(prm.tb, k1);
                     } else {
                         const uint32_t m0 = lut[cell(cur[t], e)], m1 = lut[cell(cur[t], e + 1)];
                         dense |= m0 | m1;
-                        c0 = (m0 & 15u) + (thr[m0 & 15u] < xv.x ? 1u : 0u);
-                        c1 = (m1 & 15u) + (thr[m1 & 15u] < xv.y ? 1u : 0u);
+                        c0 = (m0 & 15u) + (thr[m0 & 15u] < k0 ? 1u : 0u);
+                        c1 = (m1 & 15u) + (thr[m1 & 15u] < k1 ? 1u : 0u);
                     }
                     g = (((g << BITS) + c1) << BITS) + c0;
                 }
@@ -326,7 +329,8 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
                 if (__any_sync(0xffffffffu, dense & 0x80u)) {        // a dense cell: redo this tile's codes by search
                     g = 0;
 #pragma unroll
-                    for (int e = 7; e >= 0; --e) g = (g << BITS) + bucketize<BITS>(prm.tb, elem(cur[t], e));
+                    for (int e = 7; e >= 0; --e)
+                        g = (g << BITS) + bucketize<BITS>(prm.tb, FOLD ? fabsf(elem(cur[t], e)) : elem(cur[t], e));
                 }
             }
             grp[t] = g;
@@ -365,7 +369,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
             if (base + e < n) {
                 const float xv = load1(x + base + e);
                 store1(y + base + e, activation<ACT, T>(xv));
-                const uint32_t c = bucketize<BITS>(prm.tb, xv);
+                const uint32_t c = bucketize<BITS>(prm.tb, FOLD ? fabsf(xv) : xv);
                 const int pos = e * BITS;
                 w[pos >> 5] |= c << (pos & 31);
                 if ((pos & 31) + BITS > 32) w[(pos >> 5) + 1] |= c >> (32 - (pos & 31));
@@ -390,13 +394,13 @@ int device_sm_count(cudaError_t *err);   // of the current device, cached
 constexpr size_t kLutMinIters = 8;      // below this many warp-blocks per warp the table does not pay for its expansion
 const char *fwd_iters_override();        // tuning aid: environment FEWBIT_FWD_ITERS
 
-template <int ACT, int BITS, typename T, bool LUT>
+template <int ACT, int BITS, typename T, bool LUT, bool FOLD>
 cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *packed, size_t n, cudaStream_t st) {
     cudaError_t err = cudaSuccess;
     const int sms = device_sm_count(&err);
     if (err != cudaSuccess) return err;
     constexpr size_t smem = fwd_smem_bytes<T, LUT>();
-    auto kernel = fwd_kernel<ACT, BITS, T, LUT>;
+    auto kernel = fwd_kernel<ACT, BITS, T, LUT, FOLD>;
     if constexpr (smem > 48 * 1024) {           // opt in to the large dynamic shared memory once per device
         static std::atomic<uint64_t> opted_in{0};
         int dev = 0;
@@ -435,25 +439,33 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
 
 using FwdLaunch = cudaError_t (*)(const FwdParams &, const void *, void *, uint32_t *, size_t, cudaStream_t);
 
-// Launchers of one activation: [bits - 1][dtype is bf16][use look-up table]
-struct FwdLaunchers { FwdLaunch fn[kMaxBits][2][2]; };
+// Launchers of one activation: [bits - 1][dtype is bf16][use look-up table][folded table]
+struct FwdLaunchers { FwdLaunch fn[kMaxBits][2][2][2]; };
 
-template <int ACT, int BITS>
+template <int ACT, int BITS, bool FOLD>
 constexpr void fill_fwd_launchers(FwdLaunchers &l) {
-    l.fn[BITS - 1][0][0] = launch_fwd<ACT, BITS, float, false>;
-    // 1-2 bit binary32 tables: the search is 1-3 comparisons, cheaper than the table
-    l.fn[BITS - 1][0][1] = BITS >= 3 ? launch_fwd<ACT, BITS, float, (BITS >= 3)> : launch_fwd<ACT, BITS, float, false>;
-    l.fn[BITS - 1][1][0] = launch_fwd<ACT, BITS, __nv_bfloat16, false>;
-    l.fn[BITS - 1][1][1] = launch_fwd<ACT, BITS, __nv_bfloat16, (Bf16LutPairs<BITS>::value > 0)>;
+    // 1-2 bit binary32 tables: the search is 1-3 comparisons, cheaper than the table;
+    // bfloat16: the table only where Bf16LutPairs says so
+    constexpr bool kLutF32 = BITS >= 3, kLutBf16 = Bf16LutPairs<BITS>::value > 0;
+    l.fn[BITS - 1][0][0][FOLD] = launch_fwd<ACT, BITS, float, false, FOLD>;
+    l.fn[BITS - 1][0][1][FOLD] = launch_fwd<ACT, BITS, float, kLutF32, FOLD>;
+    l.fn[BITS - 1][1][0][FOLD] = launch_fwd<ACT, BITS, __nv_bfloat16, false, FOLD>;
+    l.fn[BITS - 1][1][1][FOLD] = launch_fwd<ACT, BITS, __nv_bfloat16, kLutBf16, FOLD>;
 }
 
 template <int ACT>
 FwdLaunchers make_fwd_launchers() {
     FwdLaunchers l{};
-    fill_fwd_launchers<ACT, 1>(l);
-    fill_fwd_launchers<ACT, 2>(l);
-    fill_fwd_launchers<ACT, 3>(l);
-    fill_fwd_launchers<ACT, 4>(l);
+    fill_fwd_launchers<ACT, 1, false>(l);
+    fill_fwd_launchers<ACT, 2, false>(l);
+    fill_fwd_launchers<ACT, 3, false>(l);
+    fill_fwd_launchers<ACT, 4, false>(l);
+    if constexpr (ACT == FEWBIT_SIGMOID || ACT == FEWBIT_TANH) {       // even f': folded tables exist
+        fill_fwd_launchers<ACT, 1, true>(l);
+        fill_fwd_launchers<ACT, 2, true>(l);
+        fill_fwd_launchers<ACT, 3, true>(l);
+        fill_fwd_launchers<ACT, 4, true>(l);
+    }
     return l;
 }
 

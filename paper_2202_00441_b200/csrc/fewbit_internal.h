@@ -35,7 +35,7 @@ struct CodeRuns {
     uint32_t run[kMaxRuns];
 };
 
-void build_code_runs(const float *s, int bits, CodeRuns *bf16_runs, CodeRuns *f32_runs);
+void build_code_runs(const float *s, int bits, bool folded, CodeRuns *bf16_runs, CodeRuns *f32_runs);
 void build_bf16_thresholds(const float *s, uint32_t *s_bf16x2);
 
 }  // namespace fewbit
@@ -45,6 +45,7 @@ void build_bf16_thresholds(const float *s, uint32_t *s_bf16x2);
 struct fewbit_table {
     fewbit_act act;
     int bits;
+    int folded;                        // 1: even f', the code is the position of |x| (table on [0, B])
     double objective;                  // value of Eq. 3 reached by the solver
     float s[fewbit::kMaxLevels];       // s[0 .. K-2]
     float lev[fewbit::kMaxLevels];     // lev[0 .. K-1]

@@ -150,7 +150,9 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
         if (force[0] == 'a') use_lut = prm.runs.count != 0;               // "always"
         else if (force[0] == 'n') use_lut = false;                        // "never"
     }
-    const cudaError_t err = fwd_launchers(table->act).fn[table->bits - 1][bf16][use_lut](
+    const FwdLaunch launch = fwd_launchers(table->act).fn[table->bits - 1][bf16][use_lut][table->folded ? 1 : 0];
+    if (launch == nullptr) return FEWBIT_ERR_UNSUPPORTED;
+    const cudaError_t err = launch(
         prm, x, y, packed, n, static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) { t_last_cuda_error = static_cast<int>(err); return FEWBIT_ERR_CUDA; }
     g_launches.fetch_add(1, std::memory_order_relaxed);

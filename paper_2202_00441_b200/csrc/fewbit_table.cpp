@@ -171,11 +171,12 @@ bool valid_bits(int b) { return b >= 1 && b <= 4; }
 // Eq. 2's interval search as a table over bit patterns: the code is a step
 // function of x with at most K-1 steps, so it is constant on long runs of
 // patterns.
-void build_code_runs(const float *s, int bits, CodeRuns *bf16_runs, CodeRuns *f32_runs) {
+void build_code_runs(const float *s, int bits, bool folded, CodeRuns *bf16_runs, CodeRuns *f32_runs) {
     const int nb = (1 << bits) - 1;
+    const auto mag = [folded](float v) { return folded ? std::fabs(v) : v; };   // |NaN| stays NaN: code 0
     {   // bfloat16: exact code of every one of the 65 536 patterns
         std::vector<uint8_t> lut(1u << kCellBitsBf16);
-        for (uint32_t p = 0; p < lut.size(); ++p) lut[p] = static_cast<uint8_t>(code_of(s, nb, from_bits(p << 16)));
+        for (uint32_t p = 0; p < lut.size(); ++p) lut[p] = static_cast<uint8_t>(code_of(s, nb, mag(from_bits(p << 16))));
         encode_runs(lut, bf16_runs);
     }
     {   // binary32: per cell of 2^19 consecutive patterns, the smaller of the codes of its two
@@ -183,8 +184,8 @@ void build_code_runs(const float *s, int bits, CodeRuns *bf16_runs, CodeRuns *f3
         std::vector<uint8_t> lut(1u << kCellBitsF32);
         const int shift = 32 - kCellBitsF32;
         for (uint32_t p = 0; p < lut.size(); ++p) {
-            const unsigned a = code_of(s, nb, from_bits(p << shift));
-            const unsigned b = code_of(s, nb, from_bits((p << shift) | ((1u << shift) - 1u)));
+            const unsigned a = code_of(s, nb, mag(from_bits(p << shift)));
+            const unsigned b = code_of(s, nb, mag(from_bits((p << shift) | ((1u << shift) - 1u))));
             const unsigned lo = a < b ? a : b, hi = a < b ? b : a;
             // a cell that mixes infinity with NaNs (code 0) is dense unless K-1 <= 1
             lut[p] = static_cast<uint8_t>((hi - lo <= 1) ? lo : kCellDense);
@@ -212,8 +213,8 @@ using fewbit::kMaxLevels;
 
 extern "C" {
 
-fewbit_status fewbit_table_create_ex(fewbit_act act, int bits, double A, double B, int n_cells,
-                                     fewbit_table **out) {
+static fewbit_status solve_into_table(fewbit_act act, int bits, double A, double B, int n_cells, bool folded,
+                                      fewbit_table **out) {
     if (out == nullptr) return FEWBIT_ERR_INVALID_ARG;
     *out = nullptr;
     if (!fewbit::valid_act(act) || !fewbit::valid_bits(bits)) return FEWBIT_ERR_INVALID_ARG;
@@ -229,7 +230,8 @@ fewbit_status fewbit_table_create_ex(fewbit_act act, int bits, double A, double 
         auto *t = new fewbit_table();
         t->act = act;
         t->bits = bits;
-        t->objective = g->best_at_n[K];
+        t->folded = folded ? 1 : 0;
+        t->objective = (folded ? 2.0 : 1.0) * g->best_at_n[K];     // both half-axes
         for (int m = 0; m < kMaxLevels; ++m) { t->s[m] = std::numeric_limits<float>::infinity(); t->lev[m] = 0.0f; }
         for (int m = 1; m < K; ++m) {
             const int i = ends[m];
@@ -237,7 +239,7 @@ fewbit_status fewbit_table_create_ex(fewbit_act act, int bits, double A, double 
             t->s[m - 1] = static_cast<float>(sm);
         }
         for (int m = 0; m < K; ++m) t->lev[m] = static_cast<float>(g->level(ends[m], ends[m + 1]));   // Eq. 4
-        fewbit::build_code_runs(t->s, bits, &t->runs_bf16, &t->runs_f32);
+        fewbit::build_code_runs(t->s, bits, folded, &t->runs_bf16, &t->runs_f32);
         fewbit::build_bf16_thresholds(t->s, t->s_bf16x2);
         *out = t;
         return FEWBIT_OK;
@@ -248,6 +250,19 @@ fewbit_status fewbit_table_create_ex(fewbit_act act, int bits, double A, double 
     }
 }
 
+fewbit_status fewbit_table_create_ex(fewbit_act act, int bits, double A, double B, int n_cells,
+                                     fewbit_table **out) {
+    return solve_into_table(act, bits, A, B, n_cells, false, out);
+}
+
+fewbit_status fewbit_table_create_folded(fewbit_act act, int bits, double B, int n_cells, fewbit_table **out) {
+    if (out != nullptr) *out = nullptr;
+    if (act != FEWBIT_SIGMOID && act != FEWBIT_TANH) return FEWBIT_ERR_UNSUPPORTED;   // f' must be even
+    return solve_into_table(act, bits, 0.0, B, n_cells, true, out);
+}
+
+int fewbit_table_is_folded(const fewbit_table *table) { return table != nullptr && table->folded; }
+
 fewbit_table *fewbit_table_create(fewbit_act act, int bits) {
     fewbit_table *t = nullptr;
     if (fewbit_table_create_ex(act, bits, -8.0, 8.0, 4096, &t) != FEWBIT_OK) return nullptr;
@@ -256,8 +271,14 @@ fewbit_table *fewbit_table_create(fewbit_act act, int bits) {
 
 fewbit_status fewbit_table_from_arrays(fewbit_act act, int bits, const float *s, const float *lev,
                                        fewbit_table **out) {
+    return fewbit_table_from_arrays_ex(act, bits, s, lev, 0, out);
+}
+
+fewbit_status fewbit_table_from_arrays_ex(fewbit_act act, int bits, const float *s, const float *lev, int folded,
+                                          fewbit_table **out) {
     if (out == nullptr) return FEWBIT_ERR_INVALID_ARG;
     *out = nullptr;
+    if (folded && act != FEWBIT_SIGMOID && act != FEWBIT_TANH) return FEWBIT_ERR_UNSUPPORTED;
     if (!fewbit::valid_act(act) || !fewbit::valid_bits(bits) || s == nullptr || lev == nullptr)
         return FEWBIT_ERR_INVALID_ARG;
     const int K = 1 << bits;
@@ -269,12 +290,13 @@ fewbit_status fewbit_table_from_arrays(fewbit_act act, int bits, const float *s,
     if (t == nullptr) return FEWBIT_ERR_ALLOC;
     t->act = act;
     t->bits = bits;
+    t->folded = folded ? 1 : 0;
     t->objective = std::numeric_limits<double>::quiet_NaN();
     for (int m = 0; m < kMaxLevels; ++m) { t->s[m] = std::numeric_limits<float>::infinity(); t->lev[m] = 0.0f; }
     // +0 and -0 compare equal; store +0 so that every kernel variant sees one pattern
     for (int m = 0; m < K - 1; ++m) t->s[m] = (s[m] == 0.0f) ? 0.0f : s[m];
     for (int m = 0; m < K; ++m) t->lev[m] = lev[m];
-    fewbit::build_code_runs(t->s, bits, &t->runs_bf16, &t->runs_f32);
+    fewbit::build_code_runs(t->s, bits, folded != 0, &t->runs_bf16, &t->runs_f32);
     fewbit::build_bf16_thresholds(t->s, t->s_bf16x2);
     *out = t;
     return FEWBIT_OK;

@@ -297,6 +297,45 @@ def test_injected_table_with_equal_boundaries(table_mode):
     assert np.array_equal(np_bits(gi), gi_ref)
 
 
+@pytest.mark.parametrize("act", ["sigmoid", "tanh"])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_folded_tables(act, dtype, table_mode):
+    """Even-derivative fold: codes from |x| against the oracle, every bit width, every variant."""
+    gen = torch.Generator(device=DEV).manual_seed(21)
+    n = 3 * 2 ** 20 + 77
+    x = (torch.randn(n, generator=gen, device=DEV) * 2).to(TORCH_DT[dtype])
+    x[:6] = torch.tensor([0.0, -0.0, float("inf"), float("-inf"), float("nan"), -1e-30], device=DEV).to(TORCH_DT[dtype])
+    g = torch.randn(n, generator=gen, device=DEV).to(TORCH_DT[dtype])
+    for bits in (1, 2, 3, 4):
+        t = fb.fewbit_table_create_folded(act, bits)
+        s, lev = t.arrays()
+        x[6:6 + s.size] = torch.from_numpy(s).to(DEV).to(TORCH_DT[dtype])
+        x[40:40 + s.size] = -torch.from_numpy(s).to(DEV).to(TORCH_DT[dtype])
+        y, p = fb.fewbit_fwd(t, x)
+        gi = fb.fewbit_bwd(t, p, g)
+        torch.cuda.synchronize()
+        y_ref, p_ref = oracle.fwd(act, bits, s, np_bits(x), fold=True)
+        gi_ref = oracle.bwd(bits, lev, p_ref, np_bits(g))
+        assert np.array_equal(np_bits(p).view(np.uint32), p_ref), (act, dtype, bits)
+        assert np.array_equal(np_bits(gi).view(gi_ref.dtype), gi_ref), (act, dtype, bits)
+        ok = finite_mask(np_bits(x))
+        assert ulp_distance(np_bits(y)[ok], y_ref[ok]).max() <= 2
+
+
+def test_folded_table_at_table_variant_size():
+    """Large enough for the shared-memory code table to be chosen on its own (bf16, 4 bits)."""
+    n = 2 ** 27
+    gen = torch.Generator(device=DEV).manual_seed(22)
+    x = (torch.randn(n, generator=gen, device=DEV) * 2).bfloat16()
+    t = fb.fewbit_table_create_folded("tanh", 4)
+    s, _ = t.arrays()
+    y, p = fb.fewbit_fwd(t, x)
+    torch.cuda.synchronize()
+    for e0 in (0, 12345 * 1024, n - 8192):
+        _, p_ref = oracle.fwd("tanh", 4, s, np_bits(x[e0:e0 + 8192]), fold=True)
+        assert np.array_equal(np_bits(p[e0 // 8:e0 // 8 + 1024]).view(np.uint32), p_ref)
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_boundaries_closer_than_a_table_cell(dtype, table_mode):
     """Boundaries a few binary32 ulps apart land in one cell of the binary32 code table (the warp

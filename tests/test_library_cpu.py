@@ -148,3 +148,29 @@ def test_memory_ratio_reproduces_the_papers_accounting():
     for bits, pct in printed.items():
         saved = nonlin * (1 - fb.fewbit_packed_bytes(32, bits) / (32 * 4)) / total
         assert round(100 * saved) == pct
+
+
+@pytest.mark.parametrize("act", ["sigmoid", "tanh"])
+def test_folded_solver_matches_oracle(lib, act):
+    """Even-derivative fold (caption of Fig. 3): the library's half-axis solve equals the oracle's."""
+    for bits in (1, 2, 3, 4):
+        t = fb.fewbit_table_create_folded(act, bits)
+        assert t.folded
+        s, lev = t.arrays()
+        r = oracle.dp_solve_folded(act, bits, 8.0, 2048)
+        assert t.objective == pytest.approx(r["objective"], abs=1e-12)
+        np.testing.assert_array_equal(s, r["s"].astype(np.float32))
+        np.testing.assert_allclose(lev, r["lev"].astype(np.float32), rtol=2e-7, atol=1e-9)
+        assert (s > 0).all()
+    assert not fb.fewbit_table_create(act, 2).folded
+
+
+def test_folded_tables_need_an_even_derivative(lib):
+    for act in ("gelu", "silu", "elu", "softplus", "leaky_relu"):
+        with pytest.raises(fb.FewbitError) as e:
+            fb.fewbit_table_create_folded(act, 2)
+        assert e.value.status == 2
+    with pytest.raises(fb.FewbitError):
+        fb.fewbit_table_from_arrays("gelu", 1, [0.5], [0.1, 0.9], folded=True)
+    assert fb.fewbit_table_from_arrays("tanh", 1, [0.5], [0.9, 0.1], folded=True).folded
+    assert lib.fewbit_table_is_folded(None) == 0
