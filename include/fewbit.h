@@ -55,9 +55,11 @@ typedef enum fewbit_act {
     FEWBIT_TANH = 3,
     FEWBIT_ELU = 4,        /* x > 0 ? x : exp(x) - 1        (alpha = 1)      */
     FEWBIT_SOFTPLUS = 5,   /* log(1 + exp(x))               (beta = 1)       */
-    FEWBIT_LEAKY_RELU = 6  /* x > 0 ? x : 0.01 x                             */
+    FEWBIT_LEAKY_RELU = 6, /* x > 0 ? x : 0.01 x                             */
+    FEWBIT_RELU = 7,       /* max(x, 0); exact with 1 bit (Sec. 2)           */
+    FEWBIT_SELU = 8        /* 1.0507 (x > 0 ? x : 1.6733 (exp(x) - 1))       */
 } fewbit_act;
-#define FEWBIT_NUM_ACTS 7
+#define FEWBIT_NUM_ACTS 9
 
 typedef enum fewbit_dtype {
     FEWBIT_F32 = 0,        /* IEEE binary32                                  */

@@ -12,3 +12,4 @@ from .binding import (  # noqa: F401
     fewbit_fwd_host_static, fewbit_static_max_elements,
 )
 from . import workloads  # noqa: F401
+from .autograd import FewBitActivation, fewbit_activation  # noqa: F401

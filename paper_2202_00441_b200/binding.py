@@ -10,7 +10,8 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libfewbit.so")
 
-ACTS = {"gelu": 0, "silu": 1, "sigmoid": 2, "tanh": 3, "elu": 4, "softplus": 5, "leaky_relu": 6}
+ACTS = {"gelu": 0, "silu": 1, "sigmoid": 2, "tanh": 3, "elu": 4, "softplus": 5, "leaky_relu": 6,
+        "relu": 7, "selu": 8}
 _DTYPES = {torch.float32: 0, torch.bfloat16: 1}
 
 _lib = None

@@ -3,7 +3,7 @@
 #include "fewbit_fwd.cuh"
 
 #ifndef FEWBIT_ACT_ID
-#error "compile with -DFEWBIT_ACT_ID=<0..6>"
+#error "compile with -DFEWBIT_ACT_ID=<0..8>"
 #endif
 
 namespace fewbit {

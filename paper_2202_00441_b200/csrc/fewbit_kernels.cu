@@ -87,6 +87,8 @@ const FwdLaunchers &fwd_launchers_act3();
 const FwdLaunchers &fwd_launchers_act4();
 const FwdLaunchers &fwd_launchers_act5();
 const FwdLaunchers &fwd_launchers_act6();
+const FwdLaunchers &fwd_launchers_act7();
+const FwdLaunchers &fwd_launchers_act8();
 
 const FwdLaunchers &fwd_launchers(int act) {
     switch (act) {
@@ -96,7 +98,9 @@ const FwdLaunchers &fwd_launchers(int act) {
     case 3: return fwd_launchers_act3();
     case 4: return fwd_launchers_act4();
     case 5: return fwd_launchers_act5();
-    default: return fwd_launchers_act6();
+    case 6: return fwd_launchers_act6();
+    case 7: return fwd_launchers_act7();
+    default: return fwd_launchers_act8();
     }
 }
 

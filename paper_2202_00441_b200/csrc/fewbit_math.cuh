@@ -35,6 +35,8 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kScaleUp = 64.0f;                      // exponent offset S
 constexpr float kScaleDown = 5.421010862427522e-20f;   // 2^-64
+constexpr float kSeluScale = 1.0507009873554805f;       // lambda
+constexpr float kSeluScaleAlpha = 1.7580993408473766f;  // lambda * alpha
 
 // ---- packed binary32 pairs (sm_100: two FMAs per issued instruction) ----------
 __device__ __forceinline__ float2 splat(float c) { return make_float2(c, c); }
@@ -97,9 +99,18 @@ __device__ __forceinline__ float2 act_bf16(float2 x) {
         const float2 small = mul2(e, fma2(es, fma2(es, splat(0.33333334f), splat(-0.5f)), splat(1.0f)));
         const float2 l = make_float2(es.x < 0.0625f ? small.x : big.x, es.y < 0.0625f ? small.y : big.y);
         return fma2(l, splat(kScaleDown), relu);
-    } else {
+    } else if constexpr (ACT == FEWBIT_LEAKY_RELU) {
         const float2 m = mul2(x, splat(0.01f));
         return make_float2(fmaxf(x.x, m.x), fmaxf(x.y, m.y));
+    } else if constexpr (ACT == FEWBIT_RELU) {
+        return relu2(x);
+    } else {
+        // SELU: lambda x for x > 0, lambda alpha (e^x - 1) otherwise; e^x - 1 = 2u / (1 - u), u = tanh(x/2)
+        const float2 h = mul2(x, splat(0.5f));
+        const float2 u = make_float2(tanh_apx(h.x), tanh_apx(h.y));
+        const float2 m = mul2(mul2(add2(u, u), splat(kSeluScaleAlpha)), rcp_2(fma2(u, splat(-1.0f), splat(1.0f))));
+        const float2 p = mul2(x, splat(kSeluScale));
+        return make_float2(x.x > 0.0f ? p.x : m.x, x.y > 0.0f ? p.y : m.y);
     }
 }
 
@@ -122,8 +133,12 @@ __device__ __forceinline__ float act_f64(float xf) {
         r = x > 0.0 ? x : expm1(x);
     } else if constexpr (ACT == FEWBIT_SOFTPLUS) {
         r = fmax(x, 0.0) + log1p(exp(-fabs(x)));
-    } else {
+    } else if constexpr (ACT == FEWBIT_LEAKY_RELU) {
         r = x > 0.0 ? x : 0.01 * x;
+    } else if constexpr (ACT == FEWBIT_RELU) {
+        r = x > 0.0 ? x : 0.0;
+    } else {
+        r = 1.0507009873554804934193349852946 * (x > 0.0 ? x : 1.6732632423543772848170429916717 * expm1(x));
     }
     return static_cast<float>(r);
 }
@@ -257,6 +272,12 @@ __device__ __forceinline__ float2 act_f32(float2 x) {
     } else if constexpr (ACT == FEWBIT_LEAKY_RELU) {
         const float2 m = mul2(x, splat(0.01f));
         return make_float2(fmaxf(x.x, m.x), fmaxf(x.y, m.y));
+    } else if constexpr (ACT == FEWBIT_RELU) {
+        return relu2(x);
+    } else if constexpr (ACT == FEWBIT_SELU) {
+        const float2 m = mul2(expm1_nonpos_f32(make_float2(fminf(x.x, 0.0f), fminf(x.y, 0.0f))), splat(kSeluScaleAlpha));
+        const float2 p = mul2(x, splat(kSeluScale));
+        return make_float2(x.x > 0.0f ? p.x : m.x, x.y > 0.0f ? p.y : m.y);
     } else {
         return make_float2(act_f64<ACT>(x.x), act_f64<ACT>(x.y));
     }

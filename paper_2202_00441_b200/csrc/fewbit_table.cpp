@@ -27,6 +27,9 @@ inline double logistic(double x) {
     return e / (1.0 + e);
 }
 
+constexpr double kSeluScale = 1.0507009873554804934193349852946;
+constexpr double kSeluAlpha = 1.6732632423543772848170429916717;
+
 inline double Phi(double x) { return 0.5 * std::erfc(-x * 0.70710678118654752440); }
 inline double phi(double x) { return 0.39894228040143267794 * std::exp(-0.5 * x * x); }
 
@@ -39,6 +42,8 @@ double value(fewbit_act a, double x) {
     case FEWBIT_ELU: return x > 0.0 ? x : std::expm1(x);
     case FEWBIT_SOFTPLUS: return std::fmax(x, 0.0) + std::log1p(std::exp(-std::fabs(x)));
     case FEWBIT_LEAKY_RELU: return x > 0.0 ? x : 0.01 * x;
+    case FEWBIT_RELU: return x > 0.0 ? x : 0.0;
+    case FEWBIT_SELU: return kSeluScale * (x > 0.0 ? x : kSeluAlpha * std::expm1(x));
     }
     return std::numeric_limits<double>::quiet_NaN();
 }
@@ -52,6 +57,8 @@ double slope(fewbit_act a, double x) {
     case FEWBIT_ELU: return x > 0.0 ? 1.0 : std::exp(x);
     case FEWBIT_SOFTPLUS: return logistic(x);
     case FEWBIT_LEAKY_RELU: return x > 0.0 ? 1.0 : 0.01;
+    case FEWBIT_RELU: return x > 0.0 ? 1.0 : 0.0;
+    case FEWBIT_SELU: return kSeluScale * (x > 0.0 ? 1.0 : kSeluAlpha * std::exp(x));
     }
     return std::numeric_limits<double>::quiet_NaN();
 }

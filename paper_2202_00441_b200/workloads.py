@@ -18,7 +18,8 @@ from typing import Iterator, Sequence, Tuple
 
 import torch
 
-ACTIVATIONS = ("gelu", "silu", "sigmoid", "tanh", "elu", "softplus", "leaky_relu")
+ACTIVATIONS = ("gelu", "silu", "sigmoid", "tanh", "elu", "softplus", "leaky_relu")   # the sweep of config 5
+EXTRA_ACTIVATIONS = ("relu", "selu")                                                 # rows of Table 1 beyond it
 
 
 @dataclasses.dataclass(frozen=True)

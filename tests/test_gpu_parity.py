@@ -238,7 +238,7 @@ def test_in_place_aliasing(dtype, table_mode):
         compare_full("tanh", bits, x, g, y, p, gi, "in place")
 
 
-@pytest.mark.parametrize("act", wl.ACTIVATIONS)
+@pytest.mark.parametrize("act", wl.ACTIVATIONS + wl.EXTRA_ACTIVATIONS)
 def test_every_bf16_pattern(act, table_mode):
     """All 65 536 bfloat16 inputs: codes for every pattern (NaN and infinities
     included), y for every finite input."""
@@ -249,7 +249,7 @@ def test_every_bf16_pattern(act, table_mode):
         compare_full(act, bits, h, g, y, p, gi, f"all bf16 {act}")
 
 
-@pytest.mark.parametrize("act", wl.ACTIVATIONS)
+@pytest.mark.parametrize("act", wl.ACTIVATIONS + wl.EXTRA_ACTIVATIONS)
 def test_f32_values_around_every_boundary_and_in_the_tails(act, table_mode):
     pieces = []
     for bits in (1, 2, 3, 4):
@@ -402,3 +402,66 @@ def test_host_entry_points_match_the_oracle(dtype, pinned):
         fb.fewbit_fwd_host(t, x, y, p, ws)
         fb.fewbit_bwd_host(t, p, g, gi, ws)
         compare_full("softplus", bits, x, g, y, p, gi, f"host {dtype} k={bits}")
+
+
+# --------------------------------------------------------------------------
+# ReLU / SELU and the autograd layer
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("act", wl.EXTRA_ACTIVATIONS)
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_relu_and_selu_against_the_oracle(act, dtype):
+    gen = torch.Generator(device=DEV).manual_seed(31)
+    n = 2 ** 21 + 5
+    x = (torch.randn(n, generator=gen, device=DEV) * 2).to(TORCH_DT[dtype])
+    g = torch.randn(n, generator=gen, device=DEV).to(TORCH_DT[dtype])
+    for bits in (1, 2, 3, 4):
+        y, p, gi = run_gpu(act, bits, x, g)
+        compare_full(act, bits, x, g, y, p, gi, f"{act} k={bits} {dtype}")
+
+
+def test_one_bit_relu_layer_is_exactly_relu():
+    """Sec. 2, ReLU paragraph: one bit reproduces the derivative, so the layer's gradient equals torch's."""
+    layer = fb.FewBitActivation("relu", bits=1)
+    x = torch.randn(1 << 18, device=DEV, requires_grad=True)
+    x2 = x.detach().clone().requires_grad_(True)
+    g = torch.randn_like(x)
+    layer(x).backward(g)
+    torch.relu(x2).backward(g)
+    assert torch.equal(x.grad, x2.grad)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_autograd_layer_matches_the_oracle_and_saves_only_the_codes(dtype):
+    bits = 3
+    layer = fb.FewBitActivation("gelu", bits=bits)
+    x = (torch.randn(64, 1031, device=DEV) * 1.5).to(TORCH_DT[dtype]).requires_grad_(True)
+    saved = []
+    with torch.autograd.graph.saved_tensors_hooks(lambda t: (saved.append(t), t)[1], lambda t: t):
+        y = layer(x)
+    assert len(saved) == 1 and saved[0].numel() * 4 == fb.fewbit_packed_bytes(x.numel(), bits)
+    g = torch.randn_like(y)
+    y.backward(g)
+    s, lev = layer.table.arrays()
+    y_ref, p_ref = oracle.fwd("gelu", bits, s, np_bits(x.detach().reshape(-1)))
+    gi_ref = oracle.bwd(bits, lev, p_ref, np_bits(g.reshape(-1)))
+    assert np.array_equal(np_bits(x.grad.reshape(-1)).view(gi_ref.dtype), gi_ref)
+    assert ulp_distance(np_bits(y.detach().reshape(-1)), y_ref).max() <= 2
+
+
+def test_autograd_layer_trains_a_small_mlp():
+    """Same initialisation, same data: the 4-bit layer trains like the exact activation."""
+    xs = torch.randn(512, 32, device=DEV, generator=torch.Generator(device=DEV).manual_seed(1))
+    ys = torch.tanh(xs[:, :4].sum(1, keepdim=True)).detach()
+    final = {}
+    for name, act in (("fewbit", lambda: fb.FewBitActivation("silu", 4)), ("exact", torch.nn.SiLU)):
+        torch.manual_seed(0)
+        net = torch.nn.Sequential(torch.nn.Linear(32, 256), act(), torch.nn.Linear(256, 1)).to(DEV)
+        opt = torch.optim.SGD(net.parameters(), lr=0.05)
+        first = None
+        for _ in range(100):
+            loss = ((net(xs) - ys) ** 2).mean()
+            first = first if first is not None else loss.item()
+            opt.zero_grad(); loss.backward(); opt.step()
+        final[name] = loss.item()
+        assert loss.item() < 0.5 * first
+    assert final["fewbit"] < 1.15 * final["exact"]

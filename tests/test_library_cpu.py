@@ -11,7 +11,7 @@ import pytest
 import oracle
 import paper_2202_00441_b200 as fb
 from paper_2202_00441_b200 import build as fb_build
-from paper_2202_00441_b200.workloads import ACTIVATIONS
+from paper_2202_00441_b200.workloads import ACTIVATIONS, EXTRA_ACTIVATIONS
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -43,7 +43,7 @@ def test_packed_bytes(lib):
     assert fb.fewbit_packed_bytes(100, 0) == 0 and fb.fewbit_packed_bytes(100, 5) == 0
 
 
-@pytest.mark.parametrize("act", ACTIVATIONS)
+@pytest.mark.parametrize("act", ACTIVATIONS + EXTRA_ACTIVATIONS)
 def test_solver_matches_oracle(lib, act):
     """The library's DP (Eq. 7-9) and the oracle's are separate programmes;
     they must reach the same optimum.  Smooth f': same boundaries, levels equal
@@ -55,7 +55,7 @@ def test_solver_matches_oracle(lib, act):
         s, lev = t.arrays()
         r = oracle.dp_solve(act, bits, -8.0, 8.0, 4096)
         assert t.objective == pytest.approx(r["objective"], abs=1e-12)
-        if act == "leaky_relu":
+        if act in ("leaky_relu", "relu"):
             probe = np.linspace(-7.99, 7.99, 4001)
             q_lib = lev[np.searchsorted(s, probe.astype(np.float32), side="left")]
             q_ref = r["lev"].astype(np.float32)[np.searchsorted(r["s"].astype(np.float32), probe.astype(np.float32), side="left")]
@@ -96,7 +96,7 @@ def test_table_from_arrays_round_trip_and_validation(lib):
 def test_invalid_table_requests(lib):
     assert not lib.fewbit_table_create(0, 0)
     assert not lib.fewbit_table_create(0, 5)
-    assert not lib.fewbit_table_create(7, 2)
+    assert not lib.fewbit_table_create(9, 2)
     assert not lib.fewbit_table_create(-1, 2)
     out = ctypes.c_void_p()
     assert lib.fewbit_table_create_ex(0, 2, 1.0, 1.0, 100, ctypes.byref(out)) == 1
