@@ -65,6 +65,18 @@ def _load():
         lib.fbo_bruteforce.restype = ctypes.c_int
         lib.fbo_bruteforce.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_int,
                                        ctypes.c_int, c_ip, c_dp]
+        lib.fbo_dp_solve_w.restype = ctypes.c_int
+        lib.fbo_dp_solve_w.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_int, ctypes.c_int,
+                                       ctypes.c_int, c_dp, c_dp, c_dp, c_ip]
+        lib.fbo_bruteforce_w.restype = ctypes.c_int
+        lib.fbo_bruteforce_w.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_int, ctypes.c_int,
+                                         ctypes.c_int, c_ip, c_dp]
+        lib.fbo_loss_at.restype = ctypes.c_double
+        lib.fbo_loss_at.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_int, ctypes.c_int,
+                                    c_dp, c_dp, c_dp]
+        lib.fbo_finetune.restype = ctypes.c_int
+        lib.fbo_finetune.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_int, ctypes.c_int,
+                                     c_dp, ctypes.c_int, c_dp, c_dp]
         lib.fbo_packed_words.restype = sz
         lib.fbo_packed_words.argtypes = [sz, ctypes.c_int]
         lib.fbo_pack.restype = None
@@ -136,19 +148,24 @@ def bf16_to_f64(h) -> np.ndarray:
 # ----------------------------------------------------------------------------
 # tables (Eq. 3, 4, 7-9)
 # ----------------------------------------------------------------------------
-def dp_solve(name, bits=None, A=-8.0, B=8.0, n_cells=4096, K=None):
+WEIGHTS = {"uniform": 0, "normal": 1}
+
+
+def dp_solve(name, bits=None, A=-8.0, B=8.0, n_cells=4096, K=None, weight="uniform"):
     """Optimal K-piece constant approximation of f' on the grid (Eq. 7).
 
-    Returns a dict with ``s`` (K-1 boundaries, f64), ``lev`` (K levels, f64),
-    ``idx`` (grid indices of the boundaries) and ``objective`` (Eq. 3)."""
+    ``weight``: "uniform" (Eq. 10 on [A,B]) or "normal" (standard normal
+    density cut to [A,B]).  Returns a dict with ``s`` (K-1 boundaries, f64),
+    ``lev`` (K levels, f64), ``idx`` (grid indices of the boundaries) and
+    ``objective`` (Eq. 3)."""
     if K is None:
         K = 1 << int(bits)
     s = np.zeros(max(K - 1, 1), dtype=np.float64)
     lev = np.zeros(K, dtype=np.float64)
     idx = np.zeros(max(K - 1, 1), dtype=np.int32)
     obj = ctypes.c_double(0.0)
-    rc = _load().fbo_dp_solve(
-        _act_id(name), float(A), float(B), int(n_cells), int(K),
+    rc = _load().fbo_dp_solve_w(
+        _act_id(name), float(A), float(B), int(n_cells), int(K), WEIGHTS[weight],
         s.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
         lev.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
         ctypes.byref(obj),
@@ -170,15 +187,42 @@ def objective(name, idx, A, B, n_cells) -> float:
     return obj.value
 
 
-def bruteforce(name, K, A, B, n_cells):
+def bruteforce(name, K, A, B, n_cells, weight="uniform"):
     """Exhaustive minimiser of Eq. 3 over all boundary subsets of the grid."""
     idx = np.zeros(max(K - 1, 1), dtype=np.int32)
     obj = ctypes.c_double(0.0)
-    rc = _load().fbo_bruteforce(_act_id(name), float(A), float(B), int(n_cells), int(K),
-                                idx.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), ctypes.byref(obj))
+    rc = _load().fbo_bruteforce_w(_act_id(name), float(A), float(B), int(n_cells), int(K), WEIGHTS[weight],
+                                  idx.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), ctypes.byref(obj))
     if rc != 0:
         raise ValueError(f"fbo_bruteforce failed with {rc}")
     return {"idx": idx[:K - 1].copy(), "objective": obj.value}
+
+
+def loss_at(name, s, A=-8.0, B=8.0, weight="uniform"):
+    """Eq. 3 at arbitrary boundaries ``s`` (levels by Eq. 4); returns
+    (L, levels, gradient by Eq. 5)."""
+    s = np.ascontiguousarray(s, dtype=np.float64)
+    K = s.size + 1
+    lev = np.zeros(K, dtype=np.float64)
+    grad = np.zeros(max(K - 1, 1), dtype=np.float64)
+    c_dp = ctypes.POINTER(ctypes.c_double)
+    val = _load().fbo_loss_at(_act_id(name), float(A), float(B), WEIGHTS[weight], K, s.ctypes.data_as(c_dp),
+                              lev.ctypes.data_as(c_dp), grad.ctypes.data_as(c_dp))
+    return val, lev, grad[:K - 1]
+
+
+def finetune(name, s, A=-8.0, B=8.0, weight="uniform", max_iter=2000):
+    """Gradient descent (Eq. 5) on the boundaries, started from ``s``."""
+    s = np.array(s, dtype=np.float64)
+    K = s.size + 1
+    lev = np.zeros(K, dtype=np.float64)
+    obj = ctypes.c_double(0.0)
+    c_dp = ctypes.POINTER(ctypes.c_double)
+    it = _load().fbo_finetune(_act_id(name), float(A), float(B), WEIGHTS[weight], K, s.ctypes.data_as(c_dp),
+                              int(max_iter), lev.ctypes.data_as(c_dp), ctypes.byref(obj))
+    if it < 0:
+        raise ValueError("fbo_finetune failed")
+    return {"s": s, "lev": lev, "objective": obj.value, "iterations": it}
 
 
 # ----------------------------------------------------------------------------

@@ -17,6 +17,13 @@
  *                             (optimal levels), uniform weight Eq. 10
  *   fbo_bruteforce            Eq. 3 minimised by exhaustive search on the grid
  *   fbo_objective             Eq. 3 for a given boundary set (levels by Eq. 4)
+ *   *_w variants              the same with the weight w chosen: 0 = indicator of
+ *                             [A,B] (Eq. 10), 1 = standard normal density cut to
+ *                             [A,B] (the other practical choice named under Eq. 3)
+ *   fbo_loss_at               Eq. 3 and its gradient Eq. 5 at arbitrary (off-grid)
+ *                             boundaries, levels by Eq. 4
+ *   fbo_finetune              gradient descent on the boundaries started from the
+ *                             DP result (Sec. 3, "Dynamic programming" paragraph)
  *   fbo_fwd_*                 Listing 1 "forward": y = f(x); code = position
  *                             of x among the boundaries s (Eq. 2); only
  *                             log2(K) bits per element are kept (Sec. 2)
@@ -109,7 +116,10 @@ typedef struct {
     double *t, *W, *FW, *F2;
 } prefix_t;
 
-static int prefix_build(prefix_t *p, int act, double A, double B, int n)
+/* w(x) on [A,B]: weight 0 -> 1, weight 1 -> standard normal density */
+static double weight_at(int weight, double x) { return weight ? std_normal_pdf(x) : 1.0; }
+
+static int prefix_build(prefix_t *p, int act, double A, double B, int n, int weight)
 {
     static const double gl_x[4] = { -0.86113631159405257522, -0.33998104358485626480,
                                      0.33998104358485626480,  0.86113631159405257522 };
@@ -124,19 +134,29 @@ static int prefix_build(prefix_t *p, int act, double A, double B, int n)
     double fA = fbo_act(act, A);
     for (int i = 0; i <= n; ++i) {
         p->t[i]  = A + (B - A) * (double)i / (double)n;
-        p->W[i]  = p->t[i] - A;
-        p->FW[i] = fbo_act(act, p->t[i]) - fA;
+        if (!weight) {                      /* closed forms for w = 1 */
+            p->W[i]  = p->t[i] - A;
+            p->FW[i] = fbo_act(act, p->t[i]) - fA;
+        }
     }
     p->t[n] = B;
     p->F2[0] = 0.0;
+    if (weight) { p->W[0] = 0.0; p->FW[0] = 0.0; }
     for (int i = 0; i < n; ++i) {
         double a = p->t[i], b = p->t[i + 1];
-        double mid = 0.5 * (a + b), half = 0.5 * (b - a), acc = 0.0;
+        double mid = 0.5 * (a + b), half = 0.5 * (b - a), acc = 0.0, accw = 0.0, accfw = 0.0;
         for (int q = 0; q < 4; ++q) {
-            double d = fbo_act_deriv(act, mid + half * gl_x[q]);
-            acc += gl_w[q] * d * d;
+            double xq = mid + half * gl_x[q];
+            double d = fbo_act_deriv(act, xq), wq = weight_at(weight, xq);
+            acc += gl_w[q] * d * d * wq;
+            accw += gl_w[q] * wq;
+            accfw += gl_w[q] * d * wq;
         }
         p->F2[i + 1] = p->F2[i] + half * acc;
+        if (weight) {                       /* Eq. 9, all three by quadrature */
+            p->W[i + 1]  = p->W[i] + half * accw;
+            p->FW[i + 1] = p->FW[i] + half * accfw;
+        }
     }
     return 0;
 }
@@ -171,12 +191,21 @@ static double bin_cost(const prefix_t *p, int j, int i)
  * s_out[K-1] = t[idx], lev_out[K] by Eq. 4 with s_0 = A and s_K = B,
  * *objective = DP(n,K).  Returns 0 on success.
  */
+int fbo_dp_solve_w(int act, double A, double B, int n, int K, int weight,
+                   double *s_out, double *lev_out, double *objective, int *idx_out);
+
 int fbo_dp_solve(int act, double A, double B, int n, int K,
                  double *s_out, double *lev_out, double *objective, int *idx_out)
 {
+    return fbo_dp_solve_w(act, A, B, n, K, 0, s_out, lev_out, objective, idx_out);
+}
+
+int fbo_dp_solve_w(int act, double A, double B, int n, int K, int weight,
+                   double *s_out, double *lev_out, double *objective, int *idx_out)
+{
     if (n < 1 || K < 1 || K > n || !(A < B)) return -1;
     prefix_t p;
-    if (prefix_build(&p, act, A, B, n)) return -2;
+    if (prefix_build(&p, act, A, B, n, weight)) return -2;
     size_t stride = (size_t)(n + 1);
     double *dp  = (double *)malloc(sizeof(double) * stride * (size_t)(K + 1));
     int    *arg = (int *)malloc(sizeof(int) * stride * (size_t)(K + 1));
@@ -214,10 +243,17 @@ int fbo_dp_solve(int act, double A, double B, int n, int K,
 }
 
 /* Eq. 3 for the boundary grid indices idx[0..K-2] (levels by Eq. 4). */
+int fbo_objective_w(int act, double A, double B, int n, int K, int weight, const int *idx, double *objective);
+
 int fbo_objective(int act, double A, double B, int n, int K, const int *idx, double *objective)
 {
+    return fbo_objective_w(act, A, B, n, K, 0, idx, objective);
+}
+
+int fbo_objective_w(int act, double A, double B, int n, int K, int weight, const int *idx, double *objective)
+{
     prefix_t p;
-    if (prefix_build(&p, act, A, B, n)) return -2;
+    if (prefix_build(&p, act, A, B, n, weight)) return -2;
     double total = 0.0;
     int left = 0;
     for (int m = 0; m < K; ++m) {
@@ -236,11 +272,18 @@ int fbo_objective(int act, double A, double B, int n, int K, const int *idx, dou
  * points 1..n-1, each scored by Eq. 3 with the levels of Eq. 4.  The
  * lexicographically first minimiser is kept.  Only for tiny n.
  */
+int fbo_bruteforce_w(int act, double A, double B, int n, int K, int weight, int *idx_out, double *objective);
+
 int fbo_bruteforce(int act, double A, double B, int n, int K, int *idx_out, double *objective)
+{
+    return fbo_bruteforce_w(act, A, B, n, K, 0, idx_out, objective);
+}
+
+int fbo_bruteforce_w(int act, double A, double B, int n, int K, int weight, int *idx_out, double *objective)
 {
     if (K < 1 || K > n) return -1;
     prefix_t p;
-    if (prefix_build(&p, act, A, B, n)) return -2;
+    if (prefix_build(&p, act, A, B, n, weight)) return -2;
     int m = K - 1;
     int *c = (int *)malloc(sizeof(int) * (size_t)(m + 1));
     for (int q = 0; q < m; ++q) c[q] = q + 1;
@@ -268,6 +311,104 @@ int fbo_bruteforce(int act, double A, double B, int n, int K, int *idx_out, doub
     free(c);
     prefix_free(&p);
     return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Off-grid boundaries: Eq. 3 with the levels of Eq. 4, its gradient Eq. 5,  */
+/* and gradient descent from the DP result.                                  */
+/* ------------------------------------------------------------------------ */
+
+/* integrals of w, f' w and f'^2 w over [a,b]: 4-point Gauss-Legendre on panels no wider than 2^-8 */
+static void bin_integrals(int act, int weight, double a, double b, double *iw, double *ifw, double *if2w)
+{
+    static const double gx[4] = { -0.86113631159405257522, -0.33998104358485626480,
+                                   0.33998104358485626480,  0.86113631159405257522 };
+    static const double gw[4] = {  0.34785484513745385737,  0.65214515486254614263,
+                                   0.65214515486254614263,  0.34785484513745385737 };
+    int panels = (int)ceil((b - a) * 256.0);
+    if (panels < 1) panels = 1;
+    double h = (b - a) / panels, sw = 0.0, sfw = 0.0, sf2 = 0.0;
+    for (int k = 0; k < panels; ++k) {
+        double mid = a + (k + 0.5) * h, half = 0.5 * h;
+        for (int q = 0; q < 4; ++q) {
+            double x = mid + half * gx[q];
+            double d = fbo_act_deriv(act, x), w = weight_at(weight, x);
+            sw += gw[q] * w * half; sfw += gw[q] * d * w * half; sf2 += gw[q] * d * d * w * half;
+        }
+    }
+    *iw = sw; *ifw = sfw; *if2w = sf2;
+}
+
+/*
+ * L(s, y(s)) of Eq. 3 for K-1 increasing boundaries s in (A,B), with
+ * y_i by Eq. 4; grad_out[i] = dL/ds_i by Eq. 5:
+ *     (2 f'(s_i) - y_i - y_{i-1}) (y_i - y_{i-1}) w(s_i),
+ * y_{i-1} the level left of s_i and y_i the level right of it.
+ * lev_out (K) and grad_out (K-1) may be NULL.  Returns L, or NAN if s is not increasing.
+ */
+double fbo_loss_at(int act, double A, double B, int weight, int K, const double *s,
+                   double *lev_out, double *grad_out)
+{
+    double lev[64];
+    double total = 0.0, left = A;
+    if (K > 64) return NAN;
+    for (int m = 0; m < K; ++m) {
+        double right = (m == K - 1) ? B : s[m];
+        if (!(right > left)) return NAN;
+        double iw, ifw, if2;
+        bin_integrals(act, weight, left, right, &iw, &ifw, &if2);
+        lev[m] = ifw / iw;                                  /* Eq. 4 */
+        total += if2 - lev[m] * lev[m] * iw;                /* int (f' - y)^2 w  with the optimal y */
+        left = right;
+    }
+    if (lev_out) for (int m = 0; m < K; ++m) lev_out[m] = lev[m];
+    if (grad_out)
+        for (int i = 0; i < K - 1; ++i)
+            grad_out[i] = (2.0 * fbo_act_deriv(act, s[i]) - lev[i + 1] - lev[i]) * (lev[i + 1] - lev[i])
+                          * weight_at(weight, s[i]);
+    return total;
+}
+
+/*
+ * Gradient descent on the boundaries.  Each component of Eq. 5 is divided by the positive factor
+ * |y_i - y_{i-1}| w(s_i) it contains (a diagonal scaling: the direction is still a descent
+ * direction, and what is left is the stationarity residual 2 f'(s_i) - y_i - y_{i-1}, so flat
+ * outer bins move as fast as steep inner ones).  The step is halved until L decreases.  At most
+ * max_iter steps; stops when every scaled component is below 1e-10.  s_inout: the DP boundaries
+ * on entry, the fine-tuned ones on exit.  Returns the number of steps taken, negative on error.
+ */
+int fbo_finetune(int act, double A, double B, int weight, int K, double *s_inout, int max_iter,
+                 double *lev_out, double *objective_out)
+{
+    double g[64], lev[64], dir[64], trial[64];
+    if (K > 64) return -1;
+    double cur = fbo_loss_at(act, A, B, weight, K, s_inout, lev, g);
+    if (isnan(cur)) return -1;
+    double step = 0.25;
+    int it = 0;
+    for (; it < max_iter; ++it) {
+        double dmax = 0.0;
+        for (int i = 0; i < K - 1; ++i) {
+            double scale = fabs(lev[i + 1] - lev[i]) * weight_at(weight, s_inout[i]);
+            dir[i] = scale > 1e-300 ? g[i] / scale : 0.0;
+            if (fabs(dir[i]) > dmax) dmax = fabs(dir[i]);
+        }
+        if (dmax < 1e-10) break;
+        int moved = 0;
+        for (int half = 0; half < 60; ++half) {
+            for (int i = 0; i < K - 1; ++i) trial[i] = s_inout[i] - step * dir[i];
+            double l = fbo_loss_at(act, A, B, weight, K, trial, NULL, NULL);
+            if (!isnan(l) && l < cur) { cur = l; moved = 1; break; }
+            step *= 0.5;
+        }
+        if (!moved) break;
+        for (int i = 0; i < K - 1; ++i) s_inout[i] = trial[i];
+        fbo_loss_at(act, A, B, weight, K, s_inout, lev, g);
+        step *= 2.0;                                        /* try a longer step next time */
+    }
+    cur = fbo_loss_at(act, A, B, weight, K, s_inout, lev_out, NULL);
+    if (objective_out) *objective_out = cur;
+    return it;
 }
 
 /* ------------------------------------------------------------------------ */

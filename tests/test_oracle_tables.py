@@ -221,3 +221,81 @@ def test_folded_levels_are_means_over_the_half_axis_bins(name):
         a, b = edges[m], edges[m + 1]
         mean = (float(MP_F[name](mp.mpf(b))) - float(MP_F[name](mp.mpf(a)))) / (b - a)
         assert r["lev"][m] == pytest.approx(mean, abs=1e-12)
+
+
+# --------------------------------------------------------------------------
+# normal weight (named under Eq. 3) and gradient fine-tuning (Eq. 5)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["gelu", "sigmoid", "elu"])
+def test_normal_weight_levels_and_objective_by_quadrature(name):
+    """Eq. 4 and Eq. 3 with w = standard normal density cut to [A,B], against scipy."""
+    A, B, n, bits = -6.0, 6.0, 768, 2
+    r = oracle.dp_solve(name, bits, A, B, n, weight="normal")
+    edges = np.concatenate([[A], r["s"], [B]])
+    fprime = lambda x: float(oracle.act_deriv(name, np.array([x]))[0])
+    pdf = lambda x: float(np.exp(-0.5 * x * x) / np.sqrt(2 * np.pi))
+    total = 0.0
+    for m in range(len(edges) - 1):
+        a, b = edges[m], edges[m + 1]
+        num, _ = integrate.quad(lambda x: fprime(x) * pdf(x), a, b, epsabs=1e-14, epsrel=1e-13, limit=200)
+        den, _ = integrate.quad(pdf, a, b, epsabs=1e-14, epsrel=1e-13, limit=200)
+        assert r["lev"][m] == pytest.approx(num / den, abs=1e-10)
+        err, _ = integrate.quad(lambda x: (fprime(x) - r["lev"][m]) ** 2 * pdf(x), a, b, epsabs=1e-14, epsrel=1e-13, limit=200)
+        total += err
+    assert r["objective"] == pytest.approx(total, abs=1e-10)
+
+
+@pytest.mark.parametrize("name", ["gelu", "silu", "tanh"])
+@pytest.mark.parametrize("n,K", [(12, 3), (16, 4), (14, 5)])
+def test_normal_weight_dp_equals_bruteforce(name, n, K):
+    dp = oracle.dp_solve(name, A=-3.0, B=4.0, n_cells=n, K=K, weight="normal")
+    bf = oracle.bruteforce(name, K, -3.0, 4.0, n, weight="normal")
+    assert dp["objective"] == pytest.approx(bf["objective"], abs=1e-16, rel=1e-13)
+    assert list(dp["idx"]) == list(bf["idx"])
+
+
+def test_normal_weight_moves_the_table_towards_the_origin():
+    """With most of the weight near 0 the outer boundaries move inwards and the weighted error
+    is far below the uniform-weight error (which pays for the whole of [-8,8])."""
+    u = oracle.dp_solve("gelu", 3)
+    w = oracle.dp_solve("gelu", 3, weight="normal")
+    assert abs(w["s"][0]) < abs(u["s"][0]) and abs(w["s"][-1]) < abs(u["s"][-1])
+    assert w["objective"] < 0.25 * u["objective"]
+    np.testing.assert_allclose(w["s"], -w["s"][::-1], atol=0)
+
+
+@pytest.mark.parametrize("weight", ["uniform", "normal"])
+@pytest.mark.parametrize("name", ["gelu", "silu", "sigmoid", "softplus"])
+def test_eq5_gradient_equals_finite_differences(name, weight):
+    rng = np.random.default_rng(5)
+    s = np.sort(rng.uniform(-3, 3, 7))
+    _, _, grad = oracle.loss_at(name, s, -8.0, 8.0, weight)
+    for i in range(s.size):
+        h = 1e-4                     # truncation ~1e-9; below that the quadrature's own 1e-13 noise / h takes over
+        sp, sm = s.copy(), s.copy()
+        sp[i] += h
+        sm[i] -= h
+        fd = (oracle.loss_at(name, sp, -8.0, 8.0, weight)[0] - oracle.loss_at(name, sm, -8.0, 8.0, weight)[0]) / (2 * h)
+        assert grad[i] == pytest.approx(fd, abs=1e-8), (name, weight, i)
+
+
+def test_loss_at_grid_points_equals_the_dp_objective():
+    r = oracle.dp_solve("silu", 3, -8.0, 8.0, 1024)
+    val, lev, _ = oracle.loss_at("silu", r["s"])
+    assert val == pytest.approx(r["objective"], abs=1e-12)
+    np.testing.assert_allclose(lev, r["lev"], atol=1e-12)
+
+
+@pytest.mark.parametrize("weight", ["uniform", "normal"])
+@pytest.mark.parametrize("name", ["gelu", "silu", "tanh", "softplus"])
+def test_finetuning_reaches_a_stationary_point_below_the_dp_value(name, weight):
+    """Sec. 3: the DP result is a starting point for gradient methods.  After fine-tuning Eq. 5
+    vanishes (2 f'(s_i) = y_i + y_{i-1} to 1e-6 instead of O(h) = 4e-3) and the error is not larger."""
+    r = oracle.dp_solve(name, 3, weight=weight)
+    ft = oracle.finetune(name, r["s"], weight=weight)
+    assert ft["objective"] <= r["objective"] + 1e-15
+    assert np.abs(ft["s"] - r["s"]).max() < 2 * 16.0 / 4096        # stays within two grid cells
+    d = oracle.act_deriv(name, ft["s"])
+    resid = np.abs(2 * d - ft["lev"][1:] - ft["lev"][:-1])
+    assert resid.max() < 1e-6, resid
+    assert (np.diff(ft["s"]) > 0).all()
