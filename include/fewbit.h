@@ -119,6 +119,31 @@ FEWBIT_API fewbit_status fewbit_table_from_arrays(fewbit_act act, int bits, cons
 FEWBIT_API fewbit_status fewbit_table_create_folded(fewbit_act act, int bits, double B, int n_cells,
                                                     fewbit_table **out);
 
+/*
+ * The solver with every choice the paper leaves open (Sec. 3):
+ *   A, B           support of the weight w of Eq. 3 (folded: A must be 0);
+ *   n_cells        grid of the dynamic programme (Eq. 7);
+ *   weight         FEWBIT_WEIGHT_UNIFORM: w = 1 on [A,B] (Eq. 10);
+ *                  FEWBIT_WEIGHT_NORMAL: w = standard normal density on [A,B];
+ *   finetune_iters 0: boundaries stay on the grid; > 0: at most that many
+ *                  gradient steps on the boundaries by Eq. 5, started from the
+ *                  DP result (boundaries then leave the grid; a few dozen
+ *                  steps reach 2 f'(s_i) = y_i + y_{i-1} to ~1e-7);
+ *   folded         as fewbit_table_create_folded.
+ * The struct is read during the call only.
+ */
+#define FEWBIT_WEIGHT_UNIFORM 0
+#define FEWBIT_WEIGHT_NORMAL 1
+typedef struct fewbit_solver_options {
+    double A, B;
+    int n_cells;
+    int weight;
+    int finetune_iters;
+    int folded;
+} fewbit_solver_options;
+FEWBIT_API fewbit_status fewbit_table_create_opt(fewbit_act act, int bits, const fewbit_solver_options *opt,
+                                                 fewbit_table **out);
+
 /* fewbit_table_from_arrays with the folded flag (folded != 0: s are boundaries of |x|). */
 FEWBIT_API fewbit_status fewbit_table_from_arrays_ex(fewbit_act act, int bits, const float *s,
                                                      const float *lev, int folded, fewbit_table **out);

@@ -52,6 +52,8 @@ def load_library():
     lib.fewbit_table_create_folded.argtypes = [ci, ci, ctypes.c_double, ci, ctypes.POINTER(vp)]
     lib.fewbit_table_from_arrays_ex.restype = ci
     lib.fewbit_table_from_arrays_ex.argtypes = [ci, ci, vp, vp, ci, ctypes.POINTER(vp)]
+    lib.fewbit_table_create_opt.restype = ci
+    lib.fewbit_table_create_opt.argtypes = [ci, ci, vp, ctypes.POINTER(vp)]
     lib.fewbit_table_is_folded.restype = ci
     lib.fewbit_table_is_folded.argtypes = [vp]
     lib.fewbit_table_destroy.restype = None
@@ -143,6 +145,22 @@ def fewbit_table_create_folded(act, bits: int, B: float = 8.0, n_cells: int = 20
     out = ctypes.c_void_p()
     _check(load_library().fewbit_table_create_folded(_act_id(act), int(bits), float(B), int(n_cells),
                                                      ctypes.byref(out)), "fewbit_table_create_folded")
+    return Table(out.value or 0)
+
+
+class _SolverOptions(ctypes.Structure):
+    _fields_ = [("A", ctypes.c_double), ("B", ctypes.c_double), ("n_cells", ctypes.c_int), ("weight", ctypes.c_int),
+                ("finetune_iters", ctypes.c_int), ("folded", ctypes.c_int)]
+
+
+def fewbit_table_create_opt(act, bits: int, A: float = -8.0, B: float = 8.0, n_cells: int = 4096,
+                            weight: str = "uniform", finetune_iters: int = 0, folded: bool = False) -> Table:
+    """Solver with explicit options: weight "uniform" | "normal" (Eq. 3), gradient fine-tuning (Eq. 5)."""
+    opt = _SolverOptions(float(A), float(B), int(n_cells), {"uniform": 0, "normal": 1}[weight], int(finetune_iters),
+                         int(bool(folded)))
+    out = ctypes.c_void_p()
+    _check(load_library().fewbit_table_create_opt(_act_id(act), int(bits), ctypes.byref(opt), ctypes.byref(out)),
+           "fewbit_table_create_opt")
     return Table(out.value or 0)
 
 

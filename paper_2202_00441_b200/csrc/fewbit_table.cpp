@@ -77,7 +77,10 @@ struct Solved {
     double level(int j, int i) const { return (FW[i] - FW[j]) / (Wt[i] - Wt[j]); }
 };
 
-std::shared_ptr<const Solved> solve_grid(fewbit_act act, double A, double B, int n) {
+// the weight w of Eq. 3 on [A,B]: 1 (Eq. 10) or the standard normal density
+inline double weight_at(int weight, double x) { return weight == FEWBIT_WEIGHT_NORMAL ? phi(x) : 1.0; }
+
+std::shared_ptr<const Solved> solve_grid(fewbit_act act, double A, double B, int n, int weight) {
     auto out = std::make_shared<Solved>();
     Solved &g = *out;
     g.n = n; g.A = A; g.B = B;
@@ -93,14 +96,22 @@ std::shared_ptr<const Solved> solve_grid(fewbit_act act, double A, double B, int
     for (int i = 1; i <= n; ++i) {
         const double right = (i == n) ? B : A + (B - A) * (static_cast<double>(i) / n);
         const double c = 0.5 * (left + right), r = 0.5 * (right - left);
-        double q = 0.0;
+        double q = 0.0, qf = 0.0;
         for (int m = 0; m < 2; ++m) {
-            const double dm = slope(act, c - r * node[m]), dp = slope(act, c + r * node[m]);
-            q += wght[m] * (dm * dm + dp * dp);
+            const double xm = c - r * node[m], xp = c + r * node[m];
+            const double dm = slope(act, xm), dp = slope(act, xp);
+            const double wm = weight_at(weight, xm), wp = weight_at(weight, xp);
+            q += wght[m] * (dm * dm * wm + dp * dp * wp);
+            qf += wght[m] * (dm * wm + dp * wp);
         }
         g.F2[i] = g.F2[i - 1] + r * q;
-        g.FW[i] = value(act, right) - fA;
-        g.Wt[i] = right - A;
+        if (weight == FEWBIT_WEIGHT_NORMAL) {
+            g.FW[i] = g.FW[i - 1] + r * qf;              // no closed form: same quadrature
+            g.Wt[i] = Phi(right) - Phi(A);               // closed form
+        } else {
+            g.FW[i] = value(act, right) - fA;
+            g.Wt[i] = right - A;
+        }
         left = right;
     }
 
@@ -136,19 +147,88 @@ std::shared_ptr<const Solved> solve_grid(fewbit_act act, double A, double B, int
 }
 
 std::mutex g_cache_mutex;
-std::map<std::tuple<int, double, double, int>, std::shared_ptr<const Solved>> g_cache;
+std::map<std::tuple<int, double, double, int, int>, std::shared_ptr<const Solved>> g_cache;
 
-std::shared_ptr<const Solved> solved_for(fewbit_act act, double A, double B, int n) {
-    const auto key = std::make_tuple(static_cast<int>(act), A, B, n);
+std::shared_ptr<const Solved> solved_for(fewbit_act act, double A, double B, int n, int weight) {
+    const auto key = std::make_tuple(static_cast<int>(act), A, B, n, weight);
     {
         std::lock_guard<std::mutex> lock(g_cache_mutex);
         auto it = g_cache.find(key);
         if (it != g_cache.end()) return it->second;
     }
-    auto fresh = solve_grid(act, A, B, n);
+    auto fresh = solve_grid(act, A, B, n, weight);
     std::lock_guard<std::mutex> lock(g_cache_mutex);
     if (g_cache.size() >= 64) g_cache.clear();
     return g_cache.emplace(key, fresh).first->second;
+}
+
+// ---------------------------------------------------------------------------
+// Off-grid refinement (Sec. 3: the DP result "can be finetuned using gradient-based methods").
+// ---------------------------------------------------------------------------
+struct BinSums { double w, fw, f2w; };
+
+// integrals of w, f'w, f'^2 w over [a,b]; Gauss-Legendre (4 nodes) on panels of width <= 2^-8
+BinSums integrate_bin(fewbit_act act, int weight, double a, double b) {
+    const double node[2] = {0.33998104358485626480, 0.86113631159405257522};
+    const double wght[2] = {0.65214515486254614263, 0.34785484513745385737};
+    const int panels = std::max(1, static_cast<int>(std::ceil((b - a) * 256.0)));
+    const double h = (b - a) / panels;
+    BinSums out{0.0, 0.0, 0.0};
+    for (int k = 0; k < panels; ++k) {
+        const double c = a + (k + 0.5) * h, r = 0.5 * h;
+        for (int m = 0; m < 2; ++m)
+            for (int sgn = -1; sgn <= 1; sgn += 2) {
+                const double x = c + sgn * r * node[m];
+                const double d = slope(act, x), w = weight_at(weight, x) * wght[m] * r;
+                out.w += w; out.fw += d * w; out.f2w += d * d * w;
+            }
+    }
+    return out;
+}
+
+// Eq. 3 at boundaries s (levels by Eq. 4 into lev); grad = Eq. 5 when not null.  NaN if s is not increasing.
+double loss_at(fewbit_act act, int weight, double A, double B, int K, const double *s, double *lev, double *grad) {
+    double total = 0.0, left = A;
+    for (int m = 0; m < K; ++m) {
+        const double right = (m == K - 1) ? B : s[m];
+        if (!(right > left)) return std::numeric_limits<double>::quiet_NaN();
+        const BinSums b = integrate_bin(act, weight, left, right);
+        lev[m] = b.fw / b.w;
+        total += b.f2w - lev[m] * lev[m] * b.w;
+        left = right;
+    }
+    if (grad != nullptr)
+        for (int i = 0; i + 1 < K; ++i)
+            grad[i] = (2.0 * slope(act, s[i]) - lev[i + 1] - lev[i]) * (lev[i + 1] - lev[i]) * weight_at(weight, s[i]);
+    return total;
+}
+
+// Descent along Eq. 5 with each component divided by its positive factor |y_i - y_{i-1}| w(s_i)
+// (what remains is the stationarity residual 2 f'(s_i) - y_i - y_{i-1}); step halved until Eq. 3 decreases.
+double finetune(fewbit_act act, int weight, double A, double B, int K, double *s, double *lev, int max_iter) {
+    double grad[kMaxLevels], dir[kMaxLevels], trial[kMaxLevels], tl[kMaxLevels];
+    double cur = loss_at(act, weight, A, B, K, s, lev, grad);
+    double step = 0.25;
+    for (int it = 0; it < max_iter && !std::isnan(cur); ++it) {
+        double largest = 0.0;
+        for (int i = 0; i + 1 < K; ++i) {
+            const double scale = std::fabs(lev[i + 1] - lev[i]) * weight_at(weight, s[i]);
+            dir[i] = scale > 1e-300 ? grad[i] / scale : 0.0;
+            largest = std::max(largest, std::fabs(dir[i]));
+        }
+        if (largest < 1e-10) break;
+        bool moved = false;
+        for (int halvings = 0; halvings < 60 && !moved; ++halvings) {
+            for (int i = 0; i + 1 < K; ++i) trial[i] = s[i] - step * dir[i];
+            const double l = loss_at(act, weight, A, B, K, trial, tl, nullptr);
+            if (!std::isnan(l) && l < cur) { cur = l; moved = true; } else { step *= 0.5; }
+        }
+        if (!moved) break;
+        for (int i = 0; i + 1 < K; ++i) s[i] = trial[i];
+        loss_at(act, weight, A, B, K, s, lev, grad);
+        step *= 2.0;
+    }
+    return loss_at(act, weight, A, B, K, s, lev, nullptr);
 }
 
 // code(x) = #{ j : s[j] < x } by a plain scan (host side, table set-up only)
@@ -221,15 +301,16 @@ using fewbit::kMaxLevels;
 extern "C" {
 
 static fewbit_status solve_into_table(fewbit_act act, int bits, double A, double B, int n_cells, bool folded,
-                                      fewbit_table **out) {
+                                      fewbit_table **out, int weight = FEWBIT_WEIGHT_UNIFORM, int finetune_iters = 0) {
     if (out == nullptr) return FEWBIT_ERR_INVALID_ARG;
     *out = nullptr;
     if (!fewbit::valid_act(act) || !fewbit::valid_bits(bits)) return FEWBIT_ERR_INVALID_ARG;
     const int K = 1 << bits;
-    if (!(A < B) || !std::isfinite(A) || !std::isfinite(B) || n_cells < K || n_cells > 65536)
+    if (!(A < B) || !std::isfinite(A) || !std::isfinite(B) || n_cells < K || n_cells > 65536 || finetune_iters < 0 ||
+        (weight != FEWBIT_WEIGHT_UNIFORM && weight != FEWBIT_WEIGHT_NORMAL))
         return FEWBIT_ERR_INVALID_ARG;
     try {
-        auto g = fewbit::solved_for(act, A, B, n_cells);
+        auto g = fewbit::solved_for(act, A, B, n_cells, weight);
         // walk the argmins back from (n, K): right ends of pieces K, K-1, ..., 1
         int ends[kMaxLevels + 1];
         ends[K] = g->n;
@@ -240,12 +321,18 @@ static fewbit_status solve_into_table(fewbit_act act, int bits, double A, double
         t->folded = folded ? 1 : 0;
         t->objective = (folded ? 2.0 : 1.0) * g->best_at_n[K];     // both half-axes
         for (int m = 0; m < kMaxLevels; ++m) { t->s[m] = std::numeric_limits<float>::infinity(); t->lev[m] = 0.0f; }
+        double sd[kMaxLevels], levd[kMaxLevels];
         for (int m = 1; m < K; ++m) {
             const int i = ends[m];
-            const double sm = (i == g->n) ? B : A + (B - A) * (static_cast<double>(i) / g->n);
-            t->s[m - 1] = static_cast<float>(sm);
+            sd[m - 1] = (i == g->n) ? B : A + (B - A) * (static_cast<double>(i) / g->n);
         }
-        for (int m = 0; m < K; ++m) t->lev[m] = static_cast<float>(g->level(ends[m], ends[m + 1]));   // Eq. 4
+        for (int m = 0; m < K; ++m) levd[m] = g->level(ends[m], ends[m + 1]);                         // Eq. 4
+        if (finetune_iters > 0) {                                                                     // Eq. 5
+            const double refined = fewbit::finetune(act, weight, A, B, K, sd, levd, finetune_iters);
+            if (!std::isnan(refined)) t->objective = (folded ? 2.0 : 1.0) * refined;
+        }
+        for (int m = 1; m < K; ++m) t->s[m - 1] = static_cast<float>(sd[m - 1]);
+        for (int m = 0; m < K; ++m) t->lev[m] = static_cast<float>(levd[m]);
         fewbit::build_code_runs(t->s, bits, folded, &t->runs_bf16, &t->runs_f32);
         fewbit::build_bf16_thresholds(t->s, t->s_bf16x2);
         *out = t;
@@ -266,6 +353,17 @@ fewbit_status fewbit_table_create_folded(fewbit_act act, int bits, double B, int
     if (out != nullptr) *out = nullptr;
     if (act != FEWBIT_SIGMOID && act != FEWBIT_TANH) return FEWBIT_ERR_UNSUPPORTED;   // f' must be even
     return solve_into_table(act, bits, 0.0, B, n_cells, true, out);
+}
+
+fewbit_status fewbit_table_create_opt(fewbit_act act, int bits, const fewbit_solver_options *opt, fewbit_table **out) {
+    if (out != nullptr) *out = nullptr;
+    if (opt == nullptr) return FEWBIT_ERR_INVALID_ARG;
+    if (opt->folded) {
+        if (act != FEWBIT_SIGMOID && act != FEWBIT_TANH) return FEWBIT_ERR_UNSUPPORTED;
+        if (opt->A != 0.0) return FEWBIT_ERR_INVALID_ARG;
+    }
+    return solve_into_table(act, bits, opt->A, opt->B, opt->n_cells, opt->folded != 0, out, opt->weight,
+                            opt->finetune_iters);
 }
 
 int fewbit_table_is_folded(const fewbit_table *table) { return table != nullptr && table->folded; }

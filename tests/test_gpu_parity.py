@@ -465,3 +465,23 @@ def test_autograd_layer_trains_a_small_mlp():
         final[name] = loss.item()
         assert loss.item() < 0.5 * first
     assert final["fewbit"] < 1.15 * final["exact"]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_finetuned_normal_weight_table(dtype, table_mode):
+    """Off-grid boundaries (Eq. 5 fine-tuning, normal weight): the hot path only sees another table."""
+    gen = torch.Generator(device=DEV).manual_seed(41)
+    n = 2 ** 20 + 333
+    x = torch.randn(n, generator=gen, device=DEV).to(TORCH_DT[dtype])
+    g = torch.randn(n, generator=gen, device=DEV).to(TORCH_DT[dtype])
+    for bits in (2, 4):
+        t = fb.fewbit_table_create_opt("gelu", bits, weight="normal", finetune_iters=500)
+        s, lev = t.arrays()
+        x[:s.size] = torch.from_numpy(s).to(DEV).to(TORCH_DT[dtype])
+        y, p = fb.fewbit_fwd(t, x)
+        gi = fb.fewbit_bwd(t, p, g)
+        torch.cuda.synchronize()
+        _, p_ref = oracle.fwd("gelu", bits, s, np_bits(x))
+        gi_ref = oracle.bwd(bits, lev, p_ref, np_bits(g))
+        assert np.array_equal(np_bits(p).view(np.uint32), p_ref)
+        assert np.array_equal(np_bits(gi).view(gi_ref.dtype), gi_ref)

@@ -174,3 +174,41 @@ def test_folded_tables_need_an_even_derivative(lib):
         fb.fewbit_table_from_arrays("gelu", 1, [0.5], [0.1, 0.9], folded=True)
     assert fb.fewbit_table_from_arrays("tanh", 1, [0.5], [0.9, 0.1], folded=True).folded
     assert lib.fewbit_table_is_folded(None) == 0
+
+
+@pytest.mark.parametrize("act", ["gelu", "silu", "tanh", "softplus"])
+@pytest.mark.parametrize("weight", ["uniform", "normal"])
+def test_weight_and_finetune_options_match_oracle(lib, act, weight):
+    """Normal weight (named under Eq. 3) and Eq. 5 fine-tuning: the library's solver and the oracle's
+    reach the same grid optimum and the same stationary point."""
+    for bits in (2, 3):
+        t = fb.fewbit_table_create_opt(act, bits, weight=weight)
+        r = oracle.dp_solve(act, bits, weight=weight)
+        assert t.objective == pytest.approx(r["objective"], abs=1e-12)
+        start = r["s"]
+        if act == "tanh" and not np.array_equal(t.arrays()[0], start.astype(np.float32)):
+            start = -start[::-1]              # even f': the mirror image is the same optimum
+        np.testing.assert_array_equal(t.arrays()[0], start.astype(np.float32))
+        tf = fb.fewbit_table_create_opt(act, bits, weight=weight, finetune_iters=2000)
+        f = oracle.finetune(act, start, weight=weight)
+        assert tf.objective == pytest.approx(f["objective"], abs=1e-10)
+        assert tf.objective <= t.objective + 1e-15
+        np.testing.assert_allclose(tf.arrays()[0], f["s"], atol=1e-5)
+        np.testing.assert_allclose(tf.arrays()[1], f["lev"], atol=1e-5)
+        s64 = tf.arrays()[0].astype(np.float64)
+        lev = tf.arrays()[1].astype(np.float64)
+        resid = np.abs(2 * oracle.act_deriv(act, s64) - lev[1:] - lev[:-1])
+        assert resid.max() < 1e-5
+
+
+def test_solver_option_validation(lib):
+    with pytest.raises(fb.FewbitError) as e:
+        fb.fewbit_table_create_opt("gelu", 2, folded=True, A=0.0)
+    assert e.value.status == 2
+    with pytest.raises(fb.FewbitError):
+        fb.fewbit_table_create_opt("tanh", 2, folded=True, A=-8.0)
+    with pytest.raises(fb.FewbitError):
+        fb.fewbit_table_create_opt("tanh", 2, finetune_iters=-1)
+    t = fb.fewbit_table_create_opt("tanh", 2, A=0.0, n_cells=2048, folded=True, weight="normal", finetune_iters=200)
+    assert t.folded and (t.arrays()[0] > 0).all()
+    assert lib.fewbit_table_create_opt(0, 2, None, None) == 1
