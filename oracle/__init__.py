@@ -87,11 +87,11 @@ def _load():
             fn = getattr(lib, name)
             fn.restype = None
             fn.argtypes = [ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, sz]
-        for name in ("fbo_fwd_f32_fold", "fbo_fwd_bf16_fold"):
+        for name in ("fbo_fwd_f32_fold", "fbo_fwd_bf16_fold", "fbo_fwd_f16_fold"):
             fn = getattr(lib, name)
             fn.restype = None
             fn.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, sz]
-        for name in ("fbo_bwd_f32", "fbo_bwd_bf16"):
+        for name in ("fbo_bwd_f32", "fbo_bwd_bf16", "fbo_bwd_f16"):
             fn = getattr(lib, name)
             fn.restype = None
             fn.argtypes = [ctypes.c_int, vp, vp, vp, vp, sz]
@@ -101,6 +101,8 @@ def _load():
             fn.argtypes = [ctypes.c_int, vp, vp, sz]
         lib.fbo_f64_to_bf16_array.restype = None
         lib.fbo_f64_to_bf16_array.argtypes = [vp, vp, sz]
+        lib.fbo_f64_to_f16_array.restype = None
+        lib.fbo_f64_to_f16_array.argtypes = [vp, vp, sz]
         _lib = lib
         return lib
 
@@ -138,6 +140,14 @@ def f64_to_bf16(x) -> np.ndarray:
     y = np.empty(x.shape, dtype=np.uint16)
     _load().fbo_f64_to_bf16_array(_ptr(x), _ptr(y), x.size)
     return y
+
+
+def f64_to_f16(x) -> np.ndarray:
+    """binary64 -> IEEE binary16 (numpy float16), one round-to-nearest-even."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    y = np.empty(x.shape, dtype=np.uint16)
+    _load().fbo_f64_to_f16_array(_ptr(x), _ptr(y), x.size)
+    return y.view(np.float16)
 
 
 def bf16_to_f64(h) -> np.ndarray:
@@ -272,9 +282,9 @@ def dp_solve_folded(name, bits, B=8.0, n_cells=2048):
 def fwd(name, bits: int, s, x: np.ndarray, fold: bool = False):
     """Forward half: returns (y, packed).
 
-    ``x`` is float32, or uint16 holding bfloat16 bit patterns; ``y`` has the
-    same dtype.  ``s`` are the K-1 boundaries as binary32.  ``fold``: the code
-    is the position of |x| (table on [0, B] for an even f')."""
+    ``x`` is float32, float16, or uint16 holding bfloat16 bit patterns; ``y``
+    has the same dtype.  ``s`` are the K-1 boundaries as binary32.  ``fold``:
+    the code is the position of |x| (table on [0, B] for an even f')."""
     s, _ = _check_tables(bits, s=s)
     if s.size == 0:
         s = np.zeros(1, dtype=np.float32)
@@ -287,8 +297,10 @@ def fwd(name, bits: int, s, x: np.ndarray, fold: bool = False):
         lib.fbo_fwd_f32_fold(_act_id(name), int(bits), int(bool(fold)), _ptr(s), _ptr(x), _ptr(y), _ptr(packed), n)
     elif x.dtype == np.uint16:
         lib.fbo_fwd_bf16_fold(_act_id(name), int(bits), int(bool(fold)), _ptr(s), _ptr(x), _ptr(y), _ptr(packed), n)
+    elif x.dtype == np.float16:
+        lib.fbo_fwd_f16_fold(_act_id(name), int(bits), int(bool(fold)), _ptr(s), _ptr(x), _ptr(y), _ptr(packed), n)
     else:
-        raise TypeError("x must be float32 or uint16 (bfloat16 bits)")
+        raise TypeError("x must be float32, float16 or uint16 (bfloat16 bits)")
     return y, packed
 
 
@@ -306,6 +318,8 @@ def bwd(bits: int, lev, packed: np.ndarray, grad_out: np.ndarray, n: int | None 
         lib.fbo_bwd_f32(int(bits), _ptr(lev), _ptr(packed), _ptr(grad_out), _ptr(grad_in), n)
     elif grad_out.dtype == np.uint16:
         lib.fbo_bwd_bf16(int(bits), _ptr(lev), _ptr(packed), _ptr(grad_out), _ptr(grad_in), n)
+    elif grad_out.dtype == np.float16:
+        lib.fbo_bwd_f16(int(bits), _ptr(lev), _ptr(packed), _ptr(grad_out), _ptr(grad_in), n)
     else:
         raise TypeError("grad_out must be float32 or uint16 (bfloat16 bits)")
     return grad_in

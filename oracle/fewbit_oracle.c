@@ -443,6 +443,36 @@ double fbo_bf16_to_f64(uint16_t h)
     uint32_t u = (uint32_t)h << 16; float f; memcpy(&f, &u, 4); return (double)f;
 }
 
+/* IEEE binary16: 5 exponent bits, 10 stored mantissa bits, subnormals below 2^-14, same method. */
+uint16_t fbo_f64_to_f16(double d)
+{
+    if (isnan(d)) return 0x7e00;
+    if (isinf(d)) return d > 0 ? 0x7c00 : 0xfc00;
+    uint16_t sign = signbit(d) ? 0x8000 : 0;
+    double a = fabs(d);
+    if (a == 0.0) return sign;
+    int e = ilogb(a);
+    if (e < -14) e = -14;                        /* subnormal range: fixed spacing 2^-24 */
+    double ulp = ldexp(1.0, e - 10);
+    double r = nearbyint(a / ulp) * ulp;         /* exact scaling, nearest-even */
+    if (r >= 65520.0) return sign | 0x7c00;      /* past the largest finite value 65504 (+ half an ulp) */
+    if (r == 0.0) return sign;
+    int er = ilogb(r);
+    if (er < -14) return sign | (uint16_t)nearbyint(r / ldexp(1.0, -24));          /* subnormal */
+    uint16_t mant = (uint16_t)nearbyint(r / ldexp(1.0, er - 10)) & 0x3ff;
+    return sign | (uint16_t)((er + 15) << 10) | mant;
+}
+
+double fbo_f16_to_f64(uint16_t h)
+{
+    int e = (h >> 10) & 0x1f, m = h & 0x3ff;
+    double v;
+    if (e == 0) v = ldexp((double)m, -24);
+    else if (e == 31) v = m ? NAN : INFINITY;
+    else v = ldexp(1.0 + m / 1024.0, e - 15);
+    return (h & 0x8000) ? -v : v;
+}
+
 static float bf16_to_f32(uint16_t h)
 {
     uint32_t u = (uint32_t)h << 16; float f; memcpy(&f, &u, 4); return f;
@@ -519,6 +549,19 @@ void fbo_fwd_bf16_fold(int act, int bits, int fold, const float *s, const uint16
     }
 }
 
+void fbo_fwd_f16_fold(int act, int bits, int fold, const float *s, const uint16_t *x, uint16_t *y,
+                      uint32_t *packed, size_t n)
+{
+    int nb = (1 << bits) - 1;
+    memset(packed, 0, 4 * fbo_packed_words(n, bits));
+    for (size_t e = 0; e < n; ++e) {
+        double xd = fbo_f16_to_f64(x[e]);
+        float xf = (float)xd;                                /* exact: binary16 is a subset of binary32 */
+        y[e] = fbo_f64_to_f16(fbo_act(act, xd));
+        put_code(packed, e, bits, bucketize(s, nb, fold ? fabsf(xf) : xf));
+    }
+}
+
 void fbo_fwd_f32(int act, int bits, const float *s, const float *x, float *y,
                  uint32_t *packed, size_t n)
 {
@@ -551,6 +594,20 @@ void fbo_bwd_bf16(int bits, const float *lev, const uint32_t *packed, const uint
         volatile float p = bf16_to_f32(grad_out[e]) * lev[get_code(packed, e, bits)];
         grad_in[e] = fbo_f64_to_bf16((double)p);
     }
+}
+
+void fbo_bwd_f16(int bits, const float *lev, const uint32_t *packed, const uint16_t *grad_out,
+                 uint16_t *grad_in, size_t n)
+{
+    for (size_t e = 0; e < n; ++e) {
+        volatile float p = (float)fbo_f16_to_f64(grad_out[e]) * lev[get_code(packed, e, bits)];
+        grad_in[e] = fbo_f64_to_f16((double)p);
+    }
+}
+
+void fbo_f64_to_f16_array(const double *x, uint16_t *y, size_t n)
+{
+    for (size_t e = 0; e < n; ++e) y[e] = fbo_f64_to_f16(x[e]);
 }
 
 /* Elementwise helpers for the Python side. */

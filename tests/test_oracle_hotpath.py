@@ -291,3 +291,46 @@ def test_folded_bucketize_is_searchsorted_of_abs(bits):
     h, f = all_finite_bf16()
     _, pb = oracle.fwd("tanh", bits, s, h, fold=True)
     np.testing.assert_array_equal(oracle.unpack(pb, bits, h.size), np.searchsorted(s, np.abs(f), side="left"))
+
+
+# --------------------------------------------------------------------------
+# IEEE binary16 storage
+# --------------------------------------------------------------------------
+def test_f16_rounding_against_numpy_and_exact_rationals():
+    """numpy converts binary64 -> float16 with one correct rounding; ties and the subnormal /
+    overflow edges are checked against exact rational arithmetic as well."""
+    xs = np.concatenate([RNG.standard_normal(20000) * 3, RNG.standard_normal(5000) * 1e-6, RNG.standard_normal(5000) * 3e4,
+                         10.0 ** RNG.uniform(-9, 5, 5000) * RNG.choice([-1, 1], 5000)])
+    allh = np.arange(0x7c00, dtype=np.uint16).view(np.float16).astype(np.float64)
+    mids = (allh[:-1] + allh[1:]) / 2                       # every tie between neighbouring finite values
+    xs = np.concatenate([xs, mids, -mids, np.nextafter(mids, 1e9), np.nextafter(mids, -1e9),
+                         [0.0, -0.0, 65504.0, 65519.99, 65520.0, 1e9, -1e9, 2.0 ** -25, 2.0 ** -25 * 1.0000001, np.inf, -np.inf]])
+    with np.errstate(over="ignore"):
+        ref = xs.astype(np.float16)
+    got = oracle.f64_to_f16(xs)
+    np.testing.assert_array_equal(got.view(np.uint16), ref.view(np.uint16))
+    vals = [Fraction(float(v)) for v in allh]
+    for x, g in zip(mids[::97], oracle.f64_to_f16(mids[::97]).view(np.uint16)):
+        lo = int(np.searchsorted(allh, x, side="right")) - 1
+        assert vals[lo] < Fraction(float(x)) < vals[lo + 1] and Fraction(float(x)) - vals[lo] == vals[lo + 1] - Fraction(float(x))
+        assert int(g) == (lo if lo % 2 == 0 else lo + 1)     # tie -> even pattern
+
+
+def test_f16_forward_and_backward_follow_the_same_rules():
+    h = np.arange(65536, dtype=np.uint16).view(np.float16)
+    f = h.astype(np.float32)
+    fin = np.isfinite(f)
+    s = np.array([-2.390625, -0.7109375, -0.328125, 0.0, 0.328125, 0.7109375, 2.390625], dtype=np.float32)
+    y, packed = oracle.fwd("gelu", 3, s, h)
+    assert y.dtype == np.float16
+    np.testing.assert_array_equal(oracle.unpack(packed, 3, h.size)[fin], np.searchsorted(s, f[fin], side="left"))
+    ref = np.array([float(MP_F["gelu"](mp.mpf(float(v)))) for v in f[fin][::37]])
+    with np.errstate(over="ignore"):
+        np.testing.assert_array_equal(y[fin][::37].view(np.uint16), ref.astype(np.float16).view(np.uint16))
+    lev = RNG.standard_normal(8).astype(np.float32)
+    g = (RNG.standard_normal(h.size) * 10.0 ** RNG.uniform(-7, 4, h.size)).astype(np.float16)
+    gi = oracle.bwd(3, lev, packed, g)
+    codes = oracle.unpack(packed, 3, h.size)
+    with np.errstate(over="ignore"):
+        ref_gi = (g.astype(np.float32) * lev[codes]).astype(np.float64).astype(np.float16)
+    np.testing.assert_array_equal(gi.view(np.uint16), ref_gi.view(np.uint16))
