@@ -344,6 +344,9 @@ def run_ours(args, case: wl.Case, act: str):
             if wl.CONFIGS[name].name != case.name:
                 also[name] = quick_config(fb, wl.CONFIGS[name], dev)
         also["c4_folded"] = quick_config(fb, wl.C4, dev, folded=True)      # even-derivative fold: codes from |x|
+        import dataclasses
+        f16 = dataclasses.replace(wl.C3, name="c3_shape_f16_2p26", dtype="f16", shape=(1 << 26,), bits=(1, 4))
+        also["f16"] = quick_config(fb, f16, dev, reps=5)                   # IEEE binary16 storage
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:

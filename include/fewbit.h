@@ -63,7 +63,8 @@ typedef enum fewbit_act {
 
 typedef enum fewbit_dtype {
     FEWBIT_F32 = 0,        /* IEEE binary32                                  */
-    FEWBIT_BF16 = 1        /* bfloat16                                       */
+    FEWBIT_BF16 = 1,       /* bfloat16                                       */
+    FEWBIT_F16 = 2         /* IEEE binary16                                  */
 } fewbit_dtype;
 
 typedef enum fewbit_status {

@@ -24,8 +24,8 @@ def _flat_aligned(t: torch.Tensor) -> torch.Tensor:
 class _FewBitFunction(torch.autograd.Function):
     @staticmethod
     def forward(ctx, x: torch.Tensor, table: Table):
-        if x.dtype not in (torch.float32, torch.bfloat16) or not x.is_cuda:
-            raise TypeError("FewBitActivation needs a CUDA tensor of dtype float32 or bfloat16")
+        if x.dtype not in (torch.float32, torch.bfloat16, torch.float16) or not x.is_cuda:
+            raise TypeError("FewBitActivation needs a CUDA tensor of dtype float32, bfloat16 or float16")
         y, packed = fewbit_fwd(table, _flat_aligned(x))
         ctx.table = table
         ctx.save_for_backward(packed)     # bits/8 bytes per element; x itself is not kept

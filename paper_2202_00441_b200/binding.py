@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_PKG, "libfewbit.so")
 
 ACTS = {"gelu": 0, "silu": 1, "sigmoid": 2, "tanh": 3, "elu": 4, "softplus": 5, "leaky_relu": 6,
         "relu": 7, "selu": 8}
-_DTYPES = {torch.float32: 0, torch.bfloat16: 1}
+_DTYPES = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 
 _lib = None
 

@@ -17,6 +17,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -73,6 +74,32 @@ __device__ __forceinline__ void store8(__nv_bfloat16 *p, const float (&v)[8]) {
     asm volatile("st.global.v4.u32 [%4], {%0,%1,%2,%3};" :: "r"(a), "r"(b), "r"(c), "r"(d), "l"(p) : "memory");
 }
 
+__device__ __forceinline__ void load8(const __half *p, float (&v)[8]) {
+    uint32_t r[4];
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "l"(p) : "memory");
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&r[i]));   // exact widening
+        v[2 * i] = f.x;
+        v[2 * i + 1] = f.y;
+    }
+}
+
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));   // round-to-nearest-even
+    return d;
+}
+
+__device__ __forceinline__ void store8(__half *p, const float (&v)[8]) {
+    const uint32_t a = pack_f16x2(v[0], v[1]), b = pack_f16x2(v[2], v[3]);
+    const uint32_t c = pack_f16x2(v[4], v[5]), d = pack_f16x2(v[6], v[7]);
+    asm volatile("st.global.v4.u32 [%4], {%0,%1,%2,%3};" :: "r"(a), "r"(b), "r"(c), "r"(d), "l"(p) : "memory");
+}
+
+__device__ __forceinline__ float load1(const __half *p) { return __half2float(*p); }
+__device__ __forceinline__ void store1(__half *p, float v) { *p = __float2half_rn(v); }
 __device__ __forceinline__ float load1(const float *p) { return *p; }
 __device__ __forceinline__ float load1(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
 __device__ __forceinline__ void store1(float *p, float v) { *p = v; }

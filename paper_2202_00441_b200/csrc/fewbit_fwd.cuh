@@ -62,14 +62,30 @@ template <typename T, bool LUT> struct FwdCtas {
     static constexpr int value = sizeof(T) == 2 ? (LUT ? FEWBIT_LUT_CTAS_BF16 : FEWBIT_CTAS_NOLUT_BF16) : kFwdCtasPerSm;
 };
 
+template <typename T> constexpr bool kIsHalf = false;
+template <> constexpr bool kIsHalf<__half> = true;
+
 template <typename T> struct Raw;                 // the 8 elements of a lane-chunk as loaded
 template <> struct Raw<float> { float v[8]; };
 template <> struct Raw<__nv_bfloat16> { uint32_t v[4]; };
+template <> struct Raw<__half> { uint32_t v[4]; };
 
 __device__ __forceinline__ void load_raw(const float *p, Raw<float> &r) { load8(p, r.v); }
 __device__ __forceinline__ void load_raw(const __nv_bfloat16 *p, Raw<__nv_bfloat16> &r) {
     asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void load_raw(const __half *p, Raw<__half> &r) {
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]) : "l"(p) : "memory");
+}
+__device__ __forceinline__ float elem(const Raw<__half> &r, int e) {
+    const __half2 h = *reinterpret_cast<const __half2 *>(&r.v[e >> 1]);
+    return (e & 1) ? __high2float(h) : __low2float(h);
+}
+__device__ __forceinline__ uint32_t pair_bits(const Raw<__half> &r, int e) { return r.v[e >> 1]; }
+__device__ __forceinline__ uint32_t cell(const Raw<__half> &r, int e) {
+    return (e & 1) ? (r.v[e >> 1] >> 16) : (r.v[e >> 1] & 0xffffu);
 }
 __device__ __forceinline__ float elem(const Raw<float> &r, int e) { return r.v[e]; }
 __device__ __forceinline__ float elem(const Raw<__nv_bfloat16> &r, int e) {
@@ -96,6 +112,9 @@ __device__ __forceinline__ uint32_t cell(const Raw<__nv_bfloat16> &r, int e) {
 __device__ __forceinline__ void cp_async_chunk(uint32_t saddr, const __nv_bfloat16 *g) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(saddr), "l"(g) : "memory");
 }
+__device__ __forceinline__ void cp_async_chunk(uint32_t saddr, const __half *g) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(saddr), "l"(g) : "memory");
+}
 __device__ __forceinline__ void cp_async_chunk(uint32_t saddr, const float *g) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(saddr), "l"(g) : "memory");
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(saddr + 16), "l"(g + 4) : "memory");
@@ -104,6 +123,9 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 
 __device__ __forceinline__ void load_raw_shared(uint32_t saddr, Raw<__nv_bfloat16> &r) {
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]) : "r"(saddr) : "memory");
+}
+__device__ __forceinline__ void load_raw_shared(uint32_t saddr, Raw<__half> &r) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]) : "r"(saddr) : "memory");
 }
 __device__ __forceinline__ void load_raw_shared(uint32_t saddr, Raw<float> &r) {
@@ -176,35 +198,37 @@ struct FwdParams {
 // packed search: codes of the two bfloat16 elements of `x2`, low element in
 // bits 0..3, high element in bits 16..19
 // ---------------------------------------------------------------------------
+template <typename T>
 __device__ __forceinline__ uint32_t gt2(uint32_t a, uint32_t b) {          // per half: 0xffff if a > b (false for NaN)
     uint32_t r;
-    asm("set.gt.u32.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    if constexpr (sizeof(T) == 2 && !kIsHalf<T>) asm("set.gt.u32.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    else asm("set.gt.u32.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
     return r;
 }
 __device__ __forceinline__ uint32_t sel2(uint32_t m, uint32_t a, uint32_t b) { return (m & a) | (~m & b); }
 
-template <int BITS>
+template <int BITS, typename T>
 __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLevels], uint32_t x2) {
     if constexpr (BITS == 1) {
-        return gt2(x2, S[0]) & 0x00010001u;
+        return gt2<T>(x2, S[0]) & 0x00010001u;
     } else if constexpr (BITS == 2) {
-        const uint32_t m1 = gt2(x2, S[1]);
-        const uint32_t m0 = gt2(x2, sel2(m1, S[2], S[0]));
+        const uint32_t m1 = gt2<T>(x2, S[1]);
+        const uint32_t m0 = gt2<T>(x2, sel2(m1, S[2], S[0]));
         return (m1 & 0x00020002u) | (m0 & 0x00010001u);
     } else if constexpr (BITS == 3) {
-        const uint32_t m2 = gt2(x2, S[3]);
-        const uint32_t m1 = gt2(x2, sel2(m2, S[5], S[1]));
-        const uint32_t m0 = gt2(x2, sel2(m1, sel2(m2, S[6], S[2]), sel2(m2, S[4], S[0])));
+        const uint32_t m2 = gt2<T>(x2, S[3]);
+        const uint32_t m1 = gt2<T>(x2, sel2(m2, S[5], S[1]));
+        const uint32_t m0 = gt2<T>(x2, sel2(m1, sel2(m2, S[6], S[2]), sel2(m2, S[4], S[0])));
         uint32_t c = m2 & 0x00040004u;
         c |= m1 & 0x00020002u;
         return c | (m0 & 0x00010001u);
     } else {
-        const uint32_t m3 = gt2(x2, S[7]);
-        const uint32_t m2 = gt2(x2, sel2(m3, S[11], S[3]));
-        const uint32_t m1 = gt2(x2, sel2(m2, sel2(m3, S[13], S[5]), sel2(m3, S[9], S[1])));
+        const uint32_t m3 = gt2<T>(x2, S[7]);
+        const uint32_t m2 = gt2<T>(x2, sel2(m3, S[11], S[3]));
+        const uint32_t m1 = gt2<T>(x2, sel2(m2, sel2(m3, S[13], S[5]), sel2(m3, S[9], S[1])));
         const uint32_t e0 = sel2(m3, S[8], S[0]), e1 = sel2(m3, S[10], S[2]);
         const uint32_t e2 = sel2(m3, S[12], S[4]), e3 = sel2(m3, S[14], S[6]);
-        const uint32_t m0 = gt2(x2, sel2(m1, sel2(m2, e3, e1), sel2(m2, e2, e0)));
+        const uint32_t m0 = gt2<T>(x2, sel2(m1, sel2(m2, e3, e1), sel2(m2, e2, e0)));
         uint32_t c = m3 & 0x00080008u;
         c |= m2 & 0x00040004u;
         c |= m1 & 0x00020002u;
@@ -300,7 +324,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
                     if (LUT && (e / 2) < Bf16LutPairs<BITS>::value) {              // resolved at compile time (unrolled)
                         pc[e / 2] = lut[cell(cur[t], e)] + (static_cast<uint32_t>(lut[cell(cur[t], e + 1)]) << 16);
                     } else {
-                        pc[e / 2] = bucketize_bf16x2<BITS>(prm.sb2, FOLD ? (pair_bits(cur[t], e) & 0x7fff7fffu) : pair_bits(cur[t], e));
+                        pc[e / 2] = bucketize_bf16x2<BITS, T>(prm.sb2, FOLD ? (pair_bits(cur[t], e) & 0x7fff7fffu) : pair_bits(cur[t], e));
                     }
                 } else {
                     uint32_t c0, c1;
@@ -439,8 +463,8 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
 
 using FwdLaunch = cudaError_t (*)(const FwdParams &, const void *, void *, uint32_t *, size_t, cudaStream_t);
 
-// Launchers of one activation: [bits - 1][dtype is bf16][use look-up table][folded table]
-struct FwdLaunchers { FwdLaunch fn[kMaxBits][2][2][2]; };
+// Launchers of one activation: [bits - 1][dtype: f32, bf16, f16][use look-up table][folded table]
+struct FwdLaunchers { FwdLaunch fn[kMaxBits][3][2][2]; };
 
 template <int ACT, int BITS, bool FOLD>
 constexpr void fill_fwd_launchers(FwdLaunchers &l) {
@@ -451,6 +475,8 @@ constexpr void fill_fwd_launchers(FwdLaunchers &l) {
     l.fn[BITS - 1][0][1][FOLD] = launch_fwd<ACT, BITS, float, kLutF32, FOLD>;
     l.fn[BITS - 1][1][0][FOLD] = launch_fwd<ACT, BITS, __nv_bfloat16, false, FOLD>;
     l.fn[BITS - 1][1][1][FOLD] = launch_fwd<ACT, BITS, __nv_bfloat16, kLutBf16, FOLD>;
+    l.fn[BITS - 1][2][0][FOLD] = launch_fwd<ACT, BITS, __half, false, FOLD>;
+    l.fn[BITS - 1][2][1][FOLD] = launch_fwd<ACT, BITS, __half, kLutBf16, FOLD>;
 }
 
 template <int ACT>

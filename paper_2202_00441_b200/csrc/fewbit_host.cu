@@ -57,7 +57,7 @@ extern "C" {
 
 size_t fewbit_host_workspace_bytes(size_t chunk_elems, fewbit_dtype dtype, int bits) {
     using namespace fewbit;
-    if (bits < 1 || bits > kMaxBits || (dtype != FEWBIT_F32 && dtype != FEWBIT_BF16)) return 0;
+    if (bits < 1 || bits > kMaxBits || !valid_dtype(dtype)) return 0;
     const size_t chunk = round_up(std::max<size_t>(chunk_elems, 1), kChunkQuantum);
     return kStages * stage_bytes(chunk, dtype, bits);
 }
@@ -65,7 +65,7 @@ size_t fewbit_host_workspace_bytes(size_t chunk_elems, fewbit_dtype dtype, int b
 fewbit_status fewbit_fwd_host(const fewbit_table *table, const void *x_host, void *y_host, uint32_t *packed_host,
                               size_t n, fewbit_dtype dtype, void *workspace, size_t workspace_bytes) {
     using namespace fewbit;
-    if (table == nullptr || (dtype != FEWBIT_F32 && dtype != FEWBIT_BF16)) return FEWBIT_ERR_INVALID_ARG;
+    if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
     if (n == 0) return FEWBIT_OK;
     if (x_host == nullptr || y_host == nullptr || packed_host == nullptr || workspace == nullptr) return FEWBIT_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(workspace) % kSlotAlign) return FEWBIT_ERR_ALIGNMENT;
@@ -102,7 +102,7 @@ fewbit_status fewbit_fwd_host(const fewbit_table *table, const void *x_host, voi
 fewbit_status fewbit_bwd_host(const fewbit_table *table, const uint32_t *packed_host, const void *grad_out_host,
                               void *grad_in_host, size_t n, fewbit_dtype dtype, void *workspace, size_t workspace_bytes) {
     using namespace fewbit;
-    if (table == nullptr || (dtype != FEWBIT_F32 && dtype != FEWBIT_BF16)) return FEWBIT_ERR_INVALID_ARG;
+    if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
     if (n == 0) return FEWBIT_OK;
     if (packed_host == nullptr || grad_out_host == nullptr || grad_in_host == nullptr || workspace == nullptr)
         return FEWBIT_ERR_INVALID_ARG;

@@ -11,6 +11,8 @@ namespace fewbit {
 constexpr int kMaxBits = 4;
 constexpr int kMaxLevels = 1 << kMaxBits;   // K <= 16
 
+inline bool valid_dtype(int d) { return d == FEWBIT_F32 || d == FEWBIT_BF16 || d == FEWBIT_F16; }
+
 extern std::atomic<uint64_t> g_launches;     // kernels launched by the library in this process
 extern thread_local int t_last_cuda_error;   // cudaError_t behind this thread's last FEWBIT_ERR_CUDA
 }  // namespace fewbit
@@ -21,7 +23,7 @@ namespace fewbit {
 // bit pattern ("cells").  Run i covers cells [start_i, start_{i+1}) and holds
 // one byte value; entry = start | value << 24.  The forward kernel expands it
 // into shared memory.
-//   bf16 table: one cell per bfloat16 pattern (65 536 cells), value = code.
+//   bf16 / f16 table: one cell per 16-bit pattern (65 536 cells), value = code.
 //   fp32 table: one cell per top-13-bit pattern (8 192 cells), value = the
 //               smallest code m in the cell when the cell holds at most one
 //               boundary (then code(x) = m + (s[m] < x)), else kCellDense.
@@ -35,8 +37,10 @@ struct CodeRuns {
     uint32_t run[kMaxRuns];
 };
 
-void build_code_runs(const float *s, int bits, bool folded, CodeRuns *bf16_runs, CodeRuns *f32_runs);
+void build_code_runs(const float *s, int bits, bool folded, CodeRuns *bf16_runs, CodeRuns *f32_runs, CodeRuns *f16_runs);
 void build_bf16_thresholds(const float *s, uint32_t *s_bf16x2);
+void build_f16_thresholds(const float *s, uint32_t *s_f16x2);
+float f16_bits_to_float(uint32_t h);
 
 }  // namespace fewbit
 
@@ -50,6 +54,8 @@ struct fewbit_table {
     float s[fewbit::kMaxLevels];       // s[0 .. K-2]
     float lev[fewbit::kMaxLevels];     // lev[0 .. K-1]
     uint32_t s_bf16x2[fewbit::kMaxLevels];   // derived from s: largest bfloat16 <= s[j], in both halves of a word
+    uint32_t s_f16x2[fewbit::kMaxLevels];    // the same for IEEE binary16
     fewbit::CodeRuns runs_bf16;        // derived from s: the bucketize step as a look-up table
+    fewbit::CodeRuns runs_f16;
     fewbit::CodeRuns runs_f32;
 };

@@ -75,9 +75,11 @@ cudaError_t launch_bwd(const Levels &tl, const uint32_t *packed, const void *g, 
     return cudaGetLastError();
 }
 
-const BwdLaunch kBwd[kMaxBits][2] = {
-    { launch_bwd<1, float>, launch_bwd<1, __nv_bfloat16> }, { launch_bwd<2, float>, launch_bwd<2, __nv_bfloat16> },
-    { launch_bwd<3, float>, launch_bwd<3, __nv_bfloat16> }, { launch_bwd<4, float>, launch_bwd<4, __nv_bfloat16> },
+const BwdLaunch kBwd[kMaxBits][3] = {      // [bits - 1][dtype: f32, bf16, f16]
+    { launch_bwd<1, float>, launch_bwd<1, __nv_bfloat16>, launch_bwd<1, __half> },
+    { launch_bwd<2, float>, launch_bwd<2, __nv_bfloat16>, launch_bwd<2, __half> },
+    { launch_bwd<3, float>, launch_bwd<3, __nv_bfloat16>, launch_bwd<3, __half> },
+    { launch_bwd<4, float>, launch_bwd<4, __nv_bfloat16>, launch_bwd<4, __half> },
 };
 
 const FwdLaunchers &fwd_launchers_act0();
@@ -136,14 +138,17 @@ extern "C" {
 fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint32_t *packed, size_t n,
                          fewbit_dtype dtype, void *stream) {
     using namespace fewbit;
-    if (table == nullptr || (dtype != FEWBIT_F32 && dtype != FEWBIT_BF16)) return FEWBIT_ERR_INVALID_ARG;
+    if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
     if (n == 0) return FEWBIT_OK;
     if (x == nullptr || y == nullptr || packed == nullptr) return FEWBIT_ERR_INVALID_ARG;
     if (!aligned(x, 32) || !aligned(y, 32) || !aligned(packed, 16)) return FEWBIT_ERR_ALIGNMENT;
     FwdParams prm;
-    for (int m = 0; m < kMaxLevels; ++m) { prm.tb.s[m] = table->s[m]; prm.sb2[m] = table->s_bf16x2[m]; }
-    const bool bf16 = dtype == FEWBIT_BF16;
-    prm.runs = bf16 ? table->runs_bf16 : table->runs_f32;
+    const bool bf16 = dtype != FEWBIT_F32;                              // a 16-bit storage type (same kernel geometry)
+    for (int m = 0; m < kMaxLevels; ++m) {
+        prm.tb.s[m] = table->s[m];
+        prm.sb2[m] = dtype == FEWBIT_F16 ? table->s_f16x2[m] : table->s_bf16x2[m];
+    }
+    prm.runs = dtype == FEWBIT_F16 ? table->runs_f16 : (bf16 ? table->runs_bf16 : table->runs_f32);
     // the shared-memory code table pays off only when every warp of a one-wave grid gets enough work
     cudaError_t sm_err = cudaSuccess;
     const size_t slots = static_cast<size_t>(device_sm_count(&sm_err)) * (bf16 ? FwdCtas<__nv_bfloat16, true>::value : FwdCtas<float, true>::value);
@@ -154,7 +159,7 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
         if (force[0] == 'a') use_lut = prm.runs.count != 0;               // "always"
         else if (force[0] == 'n') use_lut = false;                        // "never"
     }
-    const FwdLaunch launch = fwd_launchers(table->act).fn[table->bits - 1][bf16][use_lut][table->folded ? 1 : 0];
+    const FwdLaunch launch = fwd_launchers(table->act).fn[table->bits - 1][static_cast<int>(dtype)][use_lut][table->folded ? 1 : 0];
     if (launch == nullptr) return FEWBIT_ERR_UNSUPPORTED;
     const cudaError_t err = launch(
         prm, x, y, packed, n, static_cast<cudaStream_t>(stream));
@@ -166,13 +171,13 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
 fewbit_status fewbit_bwd(const fewbit_table *table, const uint32_t *packed, const void *grad_out, void *grad_in,
                          size_t n, fewbit_dtype dtype, void *stream) {
     using namespace fewbit;
-    if (table == nullptr || (dtype != FEWBIT_F32 && dtype != FEWBIT_BF16)) return FEWBIT_ERR_INVALID_ARG;
+    if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
     if (n == 0) return FEWBIT_OK;
     if (packed == nullptr || grad_out == nullptr || grad_in == nullptr) return FEWBIT_ERR_INVALID_ARG;
     if (!aligned(grad_out, 32) || !aligned(grad_in, 32) || !aligned(packed, 16)) return FEWBIT_ERR_ALIGNMENT;
     Levels tl;
     for (int m = 0; m < kMaxLevels; ++m) tl.lev[m] = table->lev[m];
-    const cudaError_t err = kBwd[table->bits - 1][dtype == FEWBIT_BF16](
+    const cudaError_t err = kBwd[table->bits - 1][static_cast<int>(dtype)](
         tl, packed, grad_out, grad_in, n, static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) { t_last_cuda_error = static_cast<int>(err); return FEWBIT_ERR_CUDA; }
     g_launches.fetch_add(1, std::memory_order_relaxed);

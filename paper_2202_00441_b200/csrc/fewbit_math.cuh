@@ -15,11 +15,17 @@
 //                      ex2.approx.ftz never flushes them) and the factor
 //                      2^-64 is folded into the last fused multiply-add, whose
 //                      IEEE gradual underflow gives correct subnormals.
+//   T = half     : as bfloat16 where the hardware approximation is 2^-22 (ex2, rcp, lg2), with a
+//                  longer GELU fit (3.5e-5) and tanh / expm1 from ex2 instead of tanh.approx
+//                  (2^-11 is not enough for 11 significant bits).
 //   T = float    : binary32 arithmetic built on an exponential good to ~0.7 ulp
 //                  (GELU: binary64 arithmetic).
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <type_traits>
 
 #include "fewbit.h"
 
@@ -283,10 +289,43 @@ __device__ __forceinline__ float2 act_f32(float2 x) {
     }
 }
 
+// ---- binary32 evaluation for binary16 storage, two elements at a time ----------
+template <int ACT>
+__device__ __forceinline__ float2 act_f16(float2 x) {
+    if constexpr (ACT == FEWBIT_GELU) {
+        // as for bfloat16, with a 5-term fit (p = 0.38, relative error 3.5e-5; fit_coefficients.py)
+        const float2 relu = relu2(x);
+        const float2 t = abs2_from_relu(relu, x);
+        const float2 e = ex2_2(fma2(mul2(x, x), splat(-0.5f * kLog2e), splat(kScaleUp)));
+        const float2 w = rcp_2(fma2(t, splat(0.38f), splat(1.0f)));
+        float2 g = fma2(w, splat(-0.08992644399404526f), splat(0.1888723224401474f));
+        g = fma2(g, w, splat(0.09198290854692459f));
+        g = fma2(g, w, splat(0.15782848000526428f));
+        g = fma2(g, w, splat(0.1512252390384674f));
+        const float2 q = mul2(mul2(g, w), e);
+        return fma2(mul2(t, q), splat(-kScaleDown), relu);
+    } else if constexpr (ACT == FEWBIT_TANH) {
+        // |x| >= 1/32: (1 - E) / (1 + E), E = e^{-2|x|} (1 - E >= 0.06, no harmful cancellation);
+        // below: x - x^3/3 (relative error 2 x^4 / 15 < 2e-7)
+        const float2 relu = relu2(x);
+        const float2 t = abs2_from_relu(relu, x);
+        const float2 e = ex2_2(mul2(t, splat(-2.0f * kLog2e)));
+        const float2 big = mul2(fma2(e, splat(-1.0f), splat(1.0f)), rcp_2(add2(e, splat(1.0f))));
+        const float2 x2 = mul2(x, x);
+        const float2 small = fma2(mul2(x2, x), splat(-0.33333334f), x);
+        return make_float2(t.x < 0.03125f ? small.x : copysignf(big.x, x.x), t.y < 0.03125f ? small.y : copysignf(big.y, x.y));
+    } else if constexpr (ACT == FEWBIT_ELU || ACT == FEWBIT_SELU) {
+        return act_f32<ACT>(x);                     // exact-constant expm1, already good to 1-2 binary32 ulp
+    } else {
+        return act_bf16<ACT>(x);                    // ex2 / rcp / lg2 forms: hardware error 2^-22
+    }
+}
+
 // two neighbouring elements at once
 template <int ACT, typename T>
 __device__ __forceinline__ float2 activation2(float2 x) {
     if constexpr (sizeof(T) == 4) return act_f32<ACT>(x);
+    else if constexpr (std::is_same<T, __half>::value) return act_f16<ACT>(x);
     else return act_bf16<ACT>(x);
 }
 

@@ -61,7 +61,7 @@ size_t fewbit_static_max_elements(void) { return fewbit::kStaticMaxElems; }
 fewbit_status fewbit_fwd_host_static(const fewbit_table *table, const void *x_host, void *y_host,
                                      uint32_t *packed_host, size_t n, fewbit_dtype dtype, void *stream) {
     using namespace fewbit;
-    if (table == nullptr || (dtype != FEWBIT_F32 && dtype != FEWBIT_BF16)) return FEWBIT_ERR_INVALID_ARG;
+    if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
     if (n == 0) return FEWBIT_OK;
     if (x_host == nullptr || y_host == nullptr || packed_host == nullptr) return FEWBIT_ERR_INVALID_ARG;
     if (n > kStaticMaxElems) return FEWBIT_ERR_TOO_LARGE;

@@ -258,13 +258,28 @@ bool valid_bits(int b) { return b >= 1 && b <= 4; }
 // Eq. 2's interval search as a table over bit patterns: the code is a step
 // function of x with at most K-1 steps, so it is constant on long runs of
 // patterns.
-void build_code_runs(const float *s, int bits, bool folded, CodeRuns *bf16_runs, CodeRuns *f32_runs) {
+// IEEE binary16 pattern -> value
+float f16_bits_to_float(uint32_t h) {
+    const int e = (h >> 10) & 0x1f, m = h & 0x3ff;
+    float v;
+    if (e == 0) v = std::ldexp(static_cast<float>(m), -24);
+    else if (e == 31) v = m ? std::numeric_limits<float>::quiet_NaN() : std::numeric_limits<float>::infinity();
+    else v = std::ldexp(1.0f + m / 1024.0f, e - 15);
+    return (h & 0x8000u) ? -v : v;
+}
+
+void build_code_runs(const float *s, int bits, bool folded, CodeRuns *bf16_runs, CodeRuns *f32_runs, CodeRuns *f16_runs) {
     const int nb = (1 << bits) - 1;
     const auto mag = [folded](float v) { return folded ? std::fabs(v) : v; };   // |NaN| stays NaN: code 0
     {   // bfloat16: exact code of every one of the 65 536 patterns
         std::vector<uint8_t> lut(1u << kCellBitsBf16);
         for (uint32_t p = 0; p < lut.size(); ++p) lut[p] = static_cast<uint8_t>(code_of(s, nb, mag(from_bits(p << 16))));
         encode_runs(lut, bf16_runs);
+    }
+    {   // binary16: exact code of every one of the 65 536 patterns
+        std::vector<uint8_t> lut(1u << 16);
+        for (uint32_t p = 0; p < lut.size(); ++p) lut[p] = static_cast<uint8_t>(code_of(s, nb, mag(f16_bits_to_float(p))));
+        encode_runs(lut, f16_runs);
     }
     {   // binary32: per cell of 2^19 consecutive patterns, the smaller of the codes of its two
         // end points when they differ by at most one (codes are monotone across a cell)
@@ -291,6 +306,24 @@ void build_bf16_thresholds(const float *s, uint32_t *s_bf16x2) {
         uint32_t h = u >> 16;
         if ((u & 0xffffu) != 0 && (u >> 31) != 0 && !std::isnan(s[j])) h += 1;   // negative and inexact: one step further from zero
         s_bf16x2[j] = h | (h << 16);
+    }
+}
+
+// The same for IEEE binary16: the largest binary16 value not above s[j] (by bisection over the
+// 63 489 ordered finite-or-infinite patterns; -inf when s[j] is below every finite value).
+void build_f16_thresholds(const float *s, uint32_t *s_f16x2) {
+    // ordered index k in [0, 2*0x7c00]: k < 0x7c00 -> negative pattern 0x8000 | (0x7c00 - k); else positive pattern k - 0x7c00
+    const auto pattern = [](int k) -> uint32_t { return k < 0x7c00 ? (0x8000u | static_cast<uint32_t>(0x7c00 - k)) : static_cast<uint32_t>(k - 0x7c00); };
+    for (int j = 0; j < kMaxLevels; ++j) {
+        int lo = 0, hi = 2 * 0x7c00;              // pattern(lo) = -inf, pattern(hi) = +inf
+        if (std::isnan(s[j]) || !(f16_bits_to_float(pattern(hi)) > s[j])) lo = hi;   // s = +inf (unused slot)
+        while (hi - lo > 1) {                    // invariant: value(lo) <= s < value(hi)
+            const int mid = (lo + hi) / 2;
+            if (f16_bits_to_float(pattern(mid)) <= s[j]) lo = mid; else hi = mid;
+        }
+        uint32_t h = pattern(lo);
+        if (h == 0x8000u) h = 0;                  // -0 and +0 compare equal; keep one pattern
+        s_f16x2[j] = h | (h << 16);
     }
 }
 
@@ -333,8 +366,9 @@ static fewbit_status solve_into_table(fewbit_act act, int bits, double A, double
         }
         for (int m = 1; m < K; ++m) t->s[m - 1] = static_cast<float>(sd[m - 1]);
         for (int m = 0; m < K; ++m) t->lev[m] = static_cast<float>(levd[m]);
-        fewbit::build_code_runs(t->s, bits, folded, &t->runs_bf16, &t->runs_f32);
+        fewbit::build_code_runs(t->s, bits, folded, &t->runs_bf16, &t->runs_f32, &t->runs_f16);
         fewbit::build_bf16_thresholds(t->s, t->s_bf16x2);
+        fewbit::build_f16_thresholds(t->s, t->s_f16x2);
         *out = t;
         return FEWBIT_OK;
     } catch (const std::bad_alloc &) {
@@ -401,8 +435,9 @@ fewbit_status fewbit_table_from_arrays_ex(fewbit_act act, int bits, const float 
     // +0 and -0 compare equal; store +0 so that every kernel variant sees one pattern
     for (int m = 0; m < K - 1; ++m) t->s[m] = (s[m] == 0.0f) ? 0.0f : s[m];
     for (int m = 0; m < K; ++m) t->lev[m] = lev[m];
-    fewbit::build_code_runs(t->s, bits, folded != 0, &t->runs_bf16, &t->runs_f32);
+    fewbit::build_code_runs(t->s, bits, folded != 0, &t->runs_bf16, &t->runs_f32, &t->runs_f16);
     fewbit::build_bf16_thresholds(t->s, t->s_bf16x2);
+    fewbit::build_f16_thresholds(t->s, t->s_f16x2);
     *out = t;
     return FEWBIT_OK;
 }

@@ -27,7 +27,7 @@ class Case:
     name: str
     acts: Tuple[str, ...]
     bits: Tuple[int, ...]
-    dtype: str                    # "f32" | "bf16"
+    dtype: str                    # "f32" | "bf16" | "f16"
     shape: Tuple[int, ...]
     x_std: float
     g_std: float
@@ -44,7 +44,7 @@ class Case:
 
     @property
     def torch_dtype(self) -> torch.dtype:
-        return torch.float32 if self.dtype == "f32" else torch.bfloat16
+        return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[self.dtype]
 
 
 C1 = Case("c1_gelu3_f32_1m", ("gelu",), (3,), "f32", (1048576,), 1.0, 1.0, 0)
@@ -95,7 +95,7 @@ def to_numpy_bits(t: torch.Tensor):
     t = t.detach().cpu().contiguous()
     if t.dtype == torch.bfloat16:
         return t.view(torch.int16).numpy().view(np.uint16)
-    if t.dtype == torch.float32:
+    if t.dtype in (torch.float32, torch.float16):
         return t.numpy()
     if t.dtype in (torch.int32, torch.uint8):
         return t.numpy()

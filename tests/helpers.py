@@ -17,6 +17,8 @@ def ulp_distance(a: np.ndarray, b: np.ndarray) -> np.ndarray:
     (bfloat16 bit pattern) arrays."""
     if a.dtype == np.float32:
         return np.abs(ordered_int(a.view(np.uint32), 32) - ordered_int(b.view(np.uint32), 32))
+    if a.dtype == np.float16:
+        return np.abs(ordered_int(a.view(np.uint16), 16) - ordered_int(b.view(np.uint16), 16))
     assert a.dtype == np.uint16
     return np.abs(ordered_int(a, 16) - ordered_int(b, 16))
 

@@ -22,7 +22,7 @@ pytestmark = pytest.mark.gpu
 
 DEV = "cuda:0"
 GUARD = 64            # guard elements / words placed around every output buffer
-TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16}
+TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
 _POOL = ThreadPoolExecutor(max_workers=8)
 _TABLES = {}
 
@@ -85,8 +85,8 @@ def compare_block(act, bits, x_np, g_np, y_np, p_np, gi_np, what):
     s, lev = table(act, bits).arrays()
     y_ref, p_ref, gi_ref = oracle_block(act, bits, s, lev, x_np, g_np)
     assert np.array_equal(p_np[:p_ref.size], p_ref), f"{what}: packed codes differ"
-    assert np.array_equal(gi_np.view(np.uint16 if gi_np.dtype == np.uint16 else np.uint32),
-                          gi_ref.view(np.uint16 if gi_ref.dtype == np.uint16 else np.uint32)), f"{what}: grad_in differs"
+    raw = np.uint32 if gi_np.dtype == np.float32 else np.uint16
+    assert np.array_equal(gi_np.view(raw), gi_ref.view(raw)), f"{what}: grad_in differs"
     ok = finite_mask(x_np)
     d = ulp_distance(y_np[ok], y_ref[ok])
     assert d.size == 0 or d.max() <= 2, f"{what}: y off by {d.max()} ulp"
@@ -485,3 +485,53 @@ def test_finetuned_normal_weight_table(dtype, table_mode):
         gi_ref = oracle.bwd(bits, lev, p_ref, np_bits(g))
         assert np.array_equal(np_bits(p).view(np.uint32), p_ref)
         assert np.array_equal(np_bits(gi).view(gi_ref.dtype), gi_ref)
+
+
+# --------------------------------------------------------------------------
+# IEEE binary16 storage
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("act", wl.ACTIVATIONS + wl.EXTRA_ACTIVATIONS)
+def test_every_f16_pattern(act, table_mode):
+    """All 65 536 binary16 inputs: codes for every pattern, y (2 ulp of binary16) for every finite one."""
+    h = torch.arange(65536, dtype=torch.int32).to(torch.int16).view(torch.float16).to(DEV)
+    g = torch.ones_like(h)
+    for bits in (1, 3, 4):
+        y, p, gi = run_gpu(act, bits, h, g)
+        compare_full(act, bits, h, g, y, p, gi, f"all f16 {act}")
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+def test_f16_random_ragged_and_gradient_specials(bits, table_mode):
+    gen = torch.Generator(device=DEV).manual_seed(51)
+    rng = np.random.default_rng(52)
+    for n in (1, 33, 1025, 70001, 2 ** 21 + 9):
+        x = (torch.randn(n, generator=gen, device=DEV) * 2).half()
+        gf = (rng.standard_normal(n) * 10.0 ** rng.uniform(-8, 4, n)).astype(np.float16)
+        g = torch.from_numpy(gf).to(DEV)
+        y, p, gi = run_gpu("gelu", bits, x, g)
+        compare_full("gelu", bits, x, g, y, p, gi, f"f16 n={n}")
+    x = (torch.randn(300001, generator=gen, device=DEV) * 2).half()
+    g = torch.randn(300001, generator=gen, device=DEV).half()
+    t = fb.fewbit_table_create_folded("tanh", bits)
+    s, lev = t.arrays()
+    y, p = fb.fewbit_fwd(t, x)
+    gi = fb.fewbit_bwd(t, p, g)
+    torch.cuda.synchronize()
+    y_ref, p_ref = oracle.fwd("tanh", bits, s, np_bits(x), fold=True)
+    assert np.array_equal(np_bits(p).view(np.uint32), p_ref)
+    assert np.array_equal(np_bits(gi).view(np.uint16), oracle.bwd(bits, lev, p_ref, np_bits(g)).view(np.uint16))
+    assert ulp_distance(np_bits(y), y_ref).max() <= 2
+
+
+def test_f16_at_table_variant_size_and_through_autograd():
+    n = 2 ** 27
+    gen = torch.Generator(device=DEV).manual_seed(53)
+    x = (torch.randn(n, generator=gen, device=DEV) * 2).half()
+    g = torch.ones_like(x)
+    y, p, gi = run_gpu("silu", 4, x, g)
+    compare_sampled("silu", 4, x, g, y, p, gi, "f16 2^27", blocks=8, block_elems=4096, seed=1)
+    del y, p, gi, g
+    layer = fb.FewBitActivation("gelu", 2)
+    xs = x[:100000].clone().requires_grad_(True)
+    layer(xs).sum().backward()
+    assert xs.grad.dtype == torch.float16 and bool(torch.isfinite(xs.grad).all())
