@@ -185,10 +185,11 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  * FEWBIT_ERR_ALIGNMENT, FEWBIT_ERR_CUDA (launch failed).
  * The interval search has several equivalent kernel variants (binary search,
  * two-at-a-time bfloat16 search, shared-memory code table) chosen from bits,
- * dtype and n; all give identical codes.  Two environment variables exist for
+ * dtype and n; all give identical codes.  Three environment variables exist for
  * testing and tuning only: FEWBIT_FWD_TABLE = always | never | auto (use of
- * the code-table variant, default auto) and FEWBIT_FWD_ITERS = <k> (warp-blocks
- * per warp).
+ * the code-table variant, default auto), FEWBIT_FWD_ITERS = <k> (warp-blocks
+ * per warp) and FEWBIT_FWD_WARPS = <w> (warps per CTA of the variants without
+ * a code table).
  */
 FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y,
                                     uint32_t *packed, size_t n, fewbit_dtype dtype, void *stream);
@@ -286,6 +287,25 @@ FEWBIT_API int fewbit_last_cuda_error(void);
 
 /* Kernels launched by this library in this process so far (all threads). */
 FEWBIT_API uint64_t fewbit_launch_count(void);
+
+/*
+ * Accuracy scan of the binary32 evaluation of an activation (the arithmetic fewbit_fwd uses for
+ * FEWBIT_F32) against the same function evaluated in binary64 and rounded once, for the `count`
+ * input bit patterns first_pattern, first_pattern + 1, ... (first_pattern + count <= 2^32; the
+ * whole range takes a few seconds).  Non-finite inputs are skipped.  The paper has no counterpart:
+ * this is a self-check of the library's arithmetic (Sec. 2 only names the functions).
+ *
+ * result_device: DEVICE pointer to 5 uint64 words, 8-byte aligned, owned by the caller; the call
+ * clears them on `stream`, then the kernel fills them:
+ *   [0], [1], [2]  inputs whose result is 0, 1, 2 ulp from the rounded binary64 value;
+ *   [3]            inputs further away (a NaN on one side only counts here);
+ *   [4]            (largest distance, capped at 2^31 - 1) << 32 | an input pattern that has it.
+ * Asynchronous on `stream`; read the words after synchronising.
+ * Errors: INVALID_ARG (bad enum, NULL, range beyond 2^32), ALIGNMENT, CUDA.
+ */
+FEWBIT_API fewbit_status fewbit_f32_activation_scan(fewbit_act act, uint64_t first_pattern,
+                                                    uint64_t count, uint64_t *result_device,
+                                                    void *stream);
 
 #ifdef __cplusplus
 }

@@ -82,6 +82,8 @@ def load_library():
     lib.fewbit_last_cuda_error.argtypes = []
     lib.fewbit_launch_count.restype = ctypes.c_uint64
     lib.fewbit_launch_count.argtypes = []
+    lib.fewbit_f32_activation_scan.restype = ci
+    lib.fewbit_f32_activation_scan.argtypes = [ci, ctypes.c_uint64, ctypes.c_uint64, vp, vp]
     _lib = lib
     return lib
 
@@ -186,6 +188,21 @@ def fewbit_packed_bytes(n: int, bits: int) -> int:
 
 def fewbit_launch_count() -> int:
     return int(load_library().fewbit_launch_count())
+
+
+def fewbit_f32_activation_scan(act, first_pattern: int = 0, count: int = 1 << 32, device=None,
+                               stream: Optional[torch.cuda.Stream] = None) -> dict:
+    """Accuracy of the binary32 evaluation of `act` against its binary64 form over a range of input
+    bit patterns (default: all of them).  Returns {"hist": [n0, n1, n2, n_more], "max_ulp": d,
+    "worst_pattern": bits}."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    res = torch.zeros(5, dtype=torch.int64, device=device)
+    with torch.cuda.device(device):
+        _check(load_library().fewbit_f32_activation_scan(_act_id(act), int(first_pattern), int(count), res.data_ptr(),
+                                                          _stream_ptr(stream, device)), "fewbit_f32_activation_scan")
+        (stream or torch.cuda.current_stream(device)).synchronize()
+    v = [int(a) & 0xFFFFFFFFFFFFFFFF for a in res.cpu().tolist()]
+    return {"hist": v[:4], "max_ulp": v[4] >> 32, "worst_pattern": v[4] & 0xFFFFFFFF}
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream], device) -> int:

@@ -259,7 +259,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     const float *thr = reinterpret_cast<const FwdSmem *>(smem_raw + kCells)->thr;
 
     const int lane = threadIdx.x & 31;
-    constexpr size_t warps = kFwdThreads / 32;                                   // stride between a warp's warp-blocks
+    const size_t warps = blockDim.x >> 5;                                        // stride between a warp's warp-blocks (<= kFwdThreads / 32)
     const size_t cta_begin = static_cast<size_t>(blockIdx.x) * warps * iters;
     const size_t warp0 = cta_begin + (threadIdx.x >> 5);
     const size_t all_full = n / kWarpElems;
@@ -417,6 +417,7 @@ constexpr size_t fwd_smem_bytes() {
 int device_sm_count(cudaError_t *err);   // of the current device, cached
 constexpr size_t kLutMinIters = 8;      // below this many warp-blocks per warp the table does not pay for its expansion
 const char *fwd_iters_override();        // tuning aid: environment FEWBIT_FWD_ITERS
+const char *fwd_warps_override();        // tuning aid: environment FEWBIT_FWD_WARPS (variant without a table)
 
 template <int ACT, int BITS, typename T, bool LUT, bool FOLD>
 cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *packed, size_t n, cudaStream_t st) {
@@ -438,25 +439,35 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
         }
     }
     constexpr int kFwdThreads = FwdThreads<T, LUT>::value;
-    constexpr size_t warps_per_cta = kFwdThreads / 32;
+    // Without a table the CTA size is free (a warp's work does not depend on it): 16-bit types run
+    // as 4-warp CTAs, which fill and drain the SMs more evenly on inputs of a few waves.
+    size_t warps_per_cta = kFwdThreads / 32;
+    if constexpr (!LUT) {
+        if constexpr (sizeof(T) == 2) warps_per_cta = 4;
+        if (const char *w = fwd_warps_override()) {
+            const int v = atoi(w);
+            if (v >= 1 && v <= kFwdThreads / 32) warps_per_cta = static_cast<size_t>(v);
+        }
+    }
     const size_t warp_blocks = n / kWarpElems + ((n % kWarpElems) ? 1 : 0);
-    // Iterations per warp.  Without a table: short CTAs, ~8 waves over the resident slots (the
-    // block scheduler evens out SMs that run slow; the prefetch ring hides the pipeline fill), at
-    // most 4.  With a table its expansion has to be amortised: exactly one wave, every CTA resident
+    // Iterations per warp.  Without a table: two from about 1.5 waves of resident warps on (the
+    // prefetch ring then overlaps a warp's loads with its arithmetic), at most 4 (short CTAs let
+    // the block scheduler even out SMs that run slow); binary32 measured fastest with one at every
+    // size (its loads are twice as wide, and more, shorter CTAs balance better).  With a table its expansion has to be amortised: exactly one wave, every CTA resident
     // from the start (the caller only picks the table variant when that gives each warp at least
     // kLutMinIters iterations).
-    const size_t slots = static_cast<size_t>(sms) * FwdCtas<T, LUT>::value;
+    const size_t slots = static_cast<size_t>(sms) * FwdCtas<T, LUT>::value * (kFwdThreads / 32) / warps_per_cta;
     size_t iters;
     if constexpr (LUT) {
         iters = (warp_blocks + warps_per_cta * slots - 1) / (warps_per_cta * slots);
     } else {
-        iters = warp_blocks / (warps_per_cta * slots * 8);
+        iters = sizeof(T) == 2 ? warp_blocks * 2 / (warps_per_cta * slots * 3) : 1;
         iters = iters < 1 ? 1 : (iters > 4 ? 4 : iters);
     }
     if (const char *dbg = fwd_iters_override()) iters = static_cast<size_t>(atoi(dbg));
     const size_t per_cta = warps_per_cta * iters;
     const unsigned grid = static_cast<unsigned>((warp_blocks + per_cta - 1) / per_cta);
-    kernel<<<grid, kFwdThreads, smem, st>>>(prm, static_cast<const T *>(x), static_cast<T *>(y), packed, n,
+    kernel<<<grid, static_cast<unsigned>(warps_per_cta * 32), smem * warps_per_cta / (kFwdThreads / 32), st>>>(prm, static_cast<const T *>(x), static_cast<T *>(y), packed, n,
                                              static_cast<int>(iters));
     return cudaGetLastError();
 }

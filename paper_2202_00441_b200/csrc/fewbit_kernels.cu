@@ -129,6 +129,11 @@ const char *fwd_iters_override() {
     return (v && *v) ? v : nullptr;
 }
 
+const char *fwd_warps_override() {
+    static const char *v = getenv("FEWBIT_FWD_WARPS");
+    return (v && *v) ? v : nullptr;
+}
+
 inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 }  // namespace fewbit

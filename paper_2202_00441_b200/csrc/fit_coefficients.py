@@ -10,9 +10,17 @@ build or run time.
    (note (1 - w) = p t w), relative error minimised by iteratively reweighted
    least squares.  The kernel needs ~2^-10 relative accuracy.
 
+   The binary16 kernel uses the same form with p = 0.38 and five terms.
+
 2. exp for binary32 storage.
    e^r = 1 + r + r^2 Q(r) on |r| <= ln(2)/2, Q of degree 4, relative error of
    e^r minimised the same way on Chebyshev nodes.
+
+3. GELU for binary32 storage.
+   Phi(-t) exp(t^2/2) = w G(w),  w = 1/(1 + p t) with p = float32(0.2),  G of
+   degree 9 in u = w - 1/2, fitted on t in [0, 15] (w in [1/4, 1]) in the
+   Chebyshev basis, relative error minimised; printed as monomials in u with
+   the constant term split into a float32 value and the float32 remainder.
 """
 import mpmath as mp
 import numpy as np
@@ -48,10 +56,33 @@ def fit_exp_f32(deg_q=4):
     return minimax_lstsq(A, target, lambda e: e * r ** 2 / np.exp(r))
 
 
+def fit_gelu_f32(p=0.2, deg=9, centre=0.5, tmax=15.0, nodes=500):
+    from numpy.polynomial import chebyshev as C, polynomial as P
+    p = float(np.float32(p))
+    wmin = 1 / (1 + p * tmax)
+    k = np.arange(nodes)
+    z = np.cos(np.pi * (k + 0.5) / nodes)
+    w = (z + 1) / 2 * (1 - wmin) + wmin
+    t = (1 / w - 1) / p
+    g = np.array([float(mp.ncdf(-mp.mpf(tt)) * mp.exp(mp.mpf(tt) ** 2 / 2) / mp.mpf(ww)) for tt, ww in zip(t, w)])
+    c, err = minimax_lstsq(C.chebvander(z, deg) / g[:, None], np.ones_like(g), lambda e: e)
+    a, b = 2 / (1 - wmin), -(1 + wmin) / (1 - wmin)          # z = a w + b = a u + (a centre + b)
+    mono = np.zeros(1)
+    for cf in C.cheb2poly(c)[::-1]:
+        mono = P.polyadd(P.polymul(mono, [a * centre + b, a]), [cf])
+    return mono, err
+
+
 if __name__ == "__main__":
     c, err = fit_gelu_bf16()
     print("GELU bf16: p = 0.30, G(w)/w coefficients (c0..c3):", [float(np.float32(v)) for v in c],
           "max relative error %.3e" % err)
+    c, err = fit_gelu_bf16(p=0.38, terms=5)
+    print("GELU f16: p = 0.38, G(w)/w coefficients (c0..c4):", [float(v) for v in c], "max relative error %.3e" % err)
+    g, err = fit_gelu_f32()
+    c0 = np.float32(g[0])
+    print("GELU f32: p = float32(0.2), G in u = w - 1/2: c0 = %.9g + %.9g, c1..c9 =" % (c0, np.float32(g[0] - float(c0))),
+          ", ".join("%.9g" % np.float32(v) for v in g[1:]), "max relative error %.3e" % err)
     q, err = fit_exp_f32()
     print("exp f32: Q coefficients (r^0..r^4):", [float(np.float32(v)) for v in q],
           "max relative error of e^r %.3e (%.3f binary32 ulp)" % (err, err / 2 ** -24))

@@ -535,3 +535,33 @@ def test_f16_at_table_variant_size_and_through_autograd():
     xs = x[:100000].clone().requires_grad_(True)
     layer(xs).sum().backward()
     assert xs.grad.dtype == torch.float16 and bool(torch.isfinite(xs.grad).all())
+
+
+@pytest.mark.parametrize("act", wl.ACTIVATIONS + wl.EXTRA_ACTIVATIONS)
+def test_f32_arithmetic_over_all_inputs_against_binary64_on_the_device(act):
+    """Every finite binary32 input: the library's binary32 evaluation of the activation is within
+    2 ulp of the binary64 evaluation rounded once.  (Device against device: it extends the parity
+    tests above, which tie the same arithmetic to the oracle on samples, to the whole input range.)"""
+    r = fb.fewbit_f32_activation_scan(act)
+    finite = 2 * (0x7F800000)                      # patterns below the infinities, both signs
+    assert sum(r["hist"]) == finite
+    assert r["hist"][3] == 0 and r["max_ulp"] <= 2, (act, r, hex(r["worst_pattern"]))
+
+
+def test_f32_scan_agrees_with_the_oracle_on_a_range():
+    """The scan's reference (binary64 on the device) and the oracle agree on what the scan reports:
+    for a stretch of patterns, the histogram of |y - oracle| recomputed on the host from fewbit_fwd
+    matches the one the scan returns."""
+    first, count = 0xBF000000, 1 << 16              # 65 536 consecutive inputs from -0.5 downward
+    bits_ = np.arange(first, first + count, dtype=np.uint32)
+    x = torch.from_numpy(bits_.view(np.float32).copy()).to(DEV)
+    for act in ("gelu", "silu", "softplus"):
+        t = table(act, 2)
+        y, _ = fb.fewbit_fwd(t, x)
+        torch.cuda.synchronize()
+        s, _ = t.arrays()
+        y_ref, _ = oracle.fwd(act, 2, s, np_bits(x))
+        d = ulp_distance(np_bits(y), y_ref)
+        hist = [int((d == k).sum()) for k in range(3)] + [int((d > 2).sum())]
+        r = fb.fewbit_f32_activation_scan(act, first, count)
+        assert r["hist"] == hist, (act, r, hist)
