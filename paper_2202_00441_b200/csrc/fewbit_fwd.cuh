@@ -415,6 +415,13 @@ constexpr size_t fwd_smem_bytes() {
 }
 
 int device_sm_count(cudaError_t *err);   // of the current device, cached
+
+// How much arithmetic an activation costs in binary32: 0 = a few instructions (ReLU, leaky ReLU),
+// 1 = one exponential or tanh, 2 = enough to make the forward kernel issue-bound (GELU, SiLU, softplus).
+constexpr int act_weight(int act) {
+    return (act == FEWBIT_RELU || act == FEWBIT_LEAKY_RELU) ? 0
+         : (act == FEWBIT_GELU || act == FEWBIT_SILU || act == FEWBIT_SOFTPLUS) ? 2 : 1;
+}
 constexpr size_t kLutMinIters = 8;      // below this many warp-blocks per warp the table does not pay for its expansion
 const char *fwd_iters_override();        // tuning aid: environment FEWBIT_FWD_ITERS
 const char *fwd_warps_override();        // tuning aid: environment FEWBIT_FWD_WARPS (variant without a table)
@@ -453,13 +460,27 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     // Iterations per warp.  Without a table: two from about 1.5 waves of resident warps on (the
     // prefetch ring then overlaps a warp's loads with its arithmetic), at most 4 (short CTAs let
     // the block scheduler even out SMs that run slow); binary32 measured fastest with one at every
-    // size (its loads are twice as wide, and more, shorter CTAs balance better).  With a table its expansion has to be amortised: exactly one wave, every CTA resident
-    // from the start (the caller only picks the table variant when that gives each warp at least
-    // kLutMinIters iterations).
+    // size (its loads are twice as wide, and more, shorter CTAs balance better).  With the 64 KB
+    // table of the 16-bit types the expansion has to be amortised: exactly one wave, every CTA
+    // resident from the start (the caller only picks that variant when this gives each warp at
+    // least kLutMinIters iterations).
     const size_t slots = static_cast<size_t>(sms) * FwdCtas<T, LUT>::value * (kFwdThreads / 32) / warps_per_cta;
     size_t iters;
     if constexpr (LUT) {
-        iters = (warp_blocks + warps_per_cta * slots - 1) / (warps_per_cta * slots);
+        const size_t waves = (warp_blocks + warps_per_cta * slots - 1) / (warps_per_cta * slots);
+        iters = waves;
+        if constexpr (sizeof(T) == 4) {
+            // The binary32 table is 8 KB: cheap to expand, so the CTAs may be short.  Measured at
+            // 2^22 .. 2^27 elements: kernels that stay memory-bound want short CTAs (the one-wave
+            // grid loses ~15 % to imbalance), issue-bound ones want the long-lived CTAs of one wave
+            // (every CTA start is a bubble in which its SM partner cannot fill the issue slots alone).
+            constexpr int kWeight = act_weight(ACT);
+            if (kWeight < 2 || waves < kLutMinIters) {
+                iters = waves / 2;
+                const size_t cap = kWeight == 0 ? 1 : 4;
+                iters = iters < 1 ? 1 : (iters > cap ? cap : iters);
+            }
+        }
     } else {
         iters = sizeof(T) == 2 ? warp_blocks * 2 / (warps_per_cta * slots * 3) : 1;
         iters = iters < 1 ? 1 : (iters > 4 ? 4 : iters);

@@ -159,7 +159,14 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
     const size_t slots = static_cast<size_t>(device_sm_count(&sm_err)) * (bf16 ? FwdCtas<__nv_bfloat16, true>::value : FwdCtas<float, true>::value);
     if (sm_err != cudaSuccess) { t_last_cuda_error = static_cast<int>(sm_err); return FEWBIT_ERR_CUDA; }
     const size_t warps_per_cta = static_cast<size_t>(bf16 ? FwdThreads<__nv_bfloat16, true>::value : FwdThreads<float, true>::value) / 32;
-    bool use_lut = prm.runs.count != 0 && n / kWarpElems >= kLutMinIters * warps_per_cta * slots;
+    const size_t waves = n / kWarpElems / (warps_per_cta * slots);
+    bool use_lut = prm.runs.count != 0 && waves >= kLutMinIters;
+    if (!bf16 && prm.runs.count != 0) {
+        // binary32 (measured, 2^22 .. 2^27 elements): at 4 bits the table beats the 4-level search at
+        // every size; at 3 bits only on large inputs, and for the light activations never
+        const int weight = act_weight(table->act);
+        use_lut = table->bits == 4 || (table->bits == 3 && ((weight == 2 && waves >= kLutMinIters) || (weight == 1 && waves >= 24)));
+    }
     if (const char *force = getenv("FEWBIT_FWD_TABLE")) {               // testing aid, see fewbit.h
         if (force[0] == 'a') use_lut = prm.runs.count != 0;               // "always"
         else if (force[0] == 'n') use_lut = false;                        // "never"
