@@ -185,11 +185,17 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  * FEWBIT_ERR_ALIGNMENT, FEWBIT_ERR_CUDA (launch failed).
  * The interval search has several equivalent kernel variants (binary search,
  * two-at-a-time bfloat16 search, shared-memory code table) chosen from bits,
- * dtype and n; all give identical codes.  Three environment variables exist for
+ * dtype and n; all give identical codes.  On large inputs of the 16-bit types
+ * at 3-4 bits the kernel distributes its work through a set of counters in a
+ * file-scope device array (16 sets per device; nothing is allocated, but the
+ * first such call on a device creates up to 16 CUDA events, and each call
+ * enqueues a 4 KB clear ahead of the kernel).  While `stream` is being captured,
+ * or when all sets are in use by other streams, the kernel falls back to a
+ * static partition: same results, ~10 % slower.  Environment variables for
  * testing and tuning only: FEWBIT_FWD_TABLE = always | never | auto (use of
- * the code-table variant, default auto), FEWBIT_FWD_ITERS = <k> (warp-blocks
- * per warp) and FEWBIT_FWD_WARPS = <w> (warps per CTA of the variants without
- * a code table).
+ * the code-table variant, default auto), FEWBIT_FWD_QUEUE = never (static
+ * partition), FEWBIT_FWD_ITERS = <k> (warp-blocks per warp) and
+ * FEWBIT_FWD_WARPS = <w> (warps per CTA of the variants without a code table).
  */
 FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y,
                                     uint32_t *packed, size_t n, fewbit_dtype dtype, void *stream);

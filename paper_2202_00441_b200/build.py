@@ -14,7 +14,7 @@ OBJ_DIR = os.path.join(PKG, "build")
 
 # (source, object stem, extra flags); the forward kernels are instantiated once per activation
 SOURCES = [("fewbit_kernels.cu", "fewbit_kernels", []), ("fewbit_host.cu", "fewbit_host", []),
-           ("fewbit_static.cu", "fewbit_static", []), ("fewbit_scan.cu", "fewbit_scan", []),
+           ("fewbit_static.cu", "fewbit_static", []), ("fewbit_scan.cu", "fewbit_scan", []), ("fewbit_queue.cu", "fewbit_queue", []),
            ("fewbit_table.cpp", "fewbit_table", [])]
 SOURCES += [("fewbit_fwd_inst.cu", f"fewbit_fwd_act{a}", [f"-DFEWBIT_ACT_ID={a}"]) for a in range(9)]
 NVCC_FLAGS = [

@@ -192,6 +192,7 @@ struct FwdParams {
     Boundaries tb;
     uint32_t sb2[kMaxLevels];        // boundaries rounded down to bfloat16, replicated in both halves
     CodeRuns runs;
+    uint32_t *queue;                 // table variants: a leased set of zeroed work counters (dynamic distribution), or NULL (static)
 };
 
 // ---------------------------------------------------------------------------
@@ -236,16 +237,6 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
     }
 }
 
-// bfloat16: how many of the four element pairs of a lane-chunk use the look-up table when the
-// kernel has one (the rest use the packed search)
-#ifndef FEWBIT_LUT_PAIRS_K3
-#define FEWBIT_LUT_PAIRS_K3 0
-#endif
-#ifndef FEWBIT_LUT_PAIRS_K4
-#define FEWBIT_LUT_PAIRS_K4 4
-#endif
-template <int BITS> struct Bf16LutPairs { static constexpr int value = BITS == 4 ? FEWBIT_LUT_PAIRS_K4 : (BITS == 3 ? FEWBIT_LUT_PAIRS_K3 : 0); };
-
 // FOLD: the code is the position of |x| (even f', table on [0, B]); the code tables arrive already
 // built that way, the searches strip the sign first.
 template <int ACT, int BITS, typename T, bool LUT, bool FOLD>
@@ -264,9 +255,32 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     const size_t warp0 = cta_begin + (threadIdx.x >> 5);
     const size_t all_full = n / kWarpElems;
     const size_t cta_end = cta_begin + warps * iters;
-    const size_t full = all_full < cta_end ? all_full : cta_end;                 // this CTA's warp-blocks are [cta_begin, full)
-
+    // Table variants may hand out warp-blocks dynamically.  Their grid is one wave of long-lived CTAs
+    // (the table is expanded once per CTA), and with a static partition the SMs that get less
+    // bandwidth finish late: 10-14 % of the kernel time at 2^28 elements.  A warp starts with the
+    // warp-block of its global warp number and takes the next unclaimed one from a counter in global
+    // memory, two iterations ahead of use, so the atomic's latency hides behind a warp-block of work.
+    // The claims go through kQueues counters, 256 bytes apart: counter q serves the warps whose
+    // global number is congruent to q and hands out the warp-blocks congruent to q (one address
+    // alone sustains only ~0.4 G atomics per second; every SM has warps in every group, so the
+    // groups finish together).
+    const bool dynamic = LUT && prm.queue != nullptr;
+    const size_t full = dynamic ? all_full : (all_full < cta_end ? all_full : cta_end);   // static: this CTA's warp-blocks are [cta_begin, full)
+    const uint32_t global_warp = blockIdx.x * static_cast<uint32_t>(warps) + (threadIdx.x >> 5);
+    const size_t first_wb = dynamic ? global_warp : warp0;
+    auto next_after = [&](size_t wb) -> size_t {
+        if constexpr (LUT) {
+            if (dynamic) {
+                uint32_t v = 0;
+                if (lane == 0) v = atomicAdd(prm.queue + (global_warp % kQueues) * kQueueStride, 1u);
+                v = __shfl_sync(0xffffffffu, v, 0);
+                return static_cast<size_t>(gridDim.x) * warps + static_cast<size_t>(v) * kQueues + global_warp % kQueues;
+            }
+        }
+        return wb + warps;
+    };
     constexpr int kStages = LUT ? (kIsBf16 ? FEWBIT_LUT_STAGES_BF16 : 0) : FEWBIT_ASYNC_STAGES;   // 0: prefetch into registers
+    static_assert(kStages >= 0 && kStages <= 2, "the loop tracks two warp-blocks ahead");
     constexpr uint32_t kRingOffset = LUT ? (kCells + static_cast<uint32_t>(sizeof(FwdSmem)) + 127u) / 128u * 128u : 0u;
     constexpr uint32_t kChunkBytes = kLaneElems * sizeof(T);
     constexpr uint32_t kStageBytes = kTilesPerWarp * 32 * kChunkBytes;          // one warp-block
@@ -276,12 +290,14 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     // consumed, the same registers are reloaded with that tile of the warp's next warp-block, so
     // four loads per lane stay in flight while the warp computes.
     Raw<T> cur[kTilesPerWarp];
+    size_t wb = first_wb;                                           // the warp-block in hand, the one after it,
+    size_t nxt = wb < full ? next_after(wb) : full;                 // and (inside the loop) the one after that
     if constexpr (kStages > 0) {
         ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw)) + kRingOffset + (threadIdx.x >> 5) * (kStages * kStageBytes) +
                lane * kChunkBytes;
 #pragma unroll
         for (int s = 0; s < kStages; ++s) {
-            const size_t wbs = warp0 + s * warps;
+            const size_t wbs = s == 0 ? wb : nxt;
             if (wbs < full) {
                 const T *px = x + wbs * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
 #pragma unroll
@@ -290,8 +306,8 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
             }
             cp_async_commit();
         }
-    } else if (warp0 < full) {
-        const T *px = x + warp0 * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
+    } else if (wb < full) {
+        const T *px = x + wb * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
 #pragma unroll
         for (int t = 0; t < kTilesPerWarp; ++t) load_raw(px + t * kTileElems, cur[t]);
     }
@@ -300,11 +316,12 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         if (threadIdx.x < kMaxLevels) sm.thr[threadIdx.x] = prm.tb.s[threadIdx.x];
         expand_runs<kCells, kFwdThreads>(prm.runs, lut, sm);
     }
-    for (size_t wb = warp0; wb < full; wb += warps) {
+    while (wb < full) {
         const size_t base = wb * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
         T *py = y + base;
-        const T *px_next = x + base + warps * kWarpElems;
-        const bool more = wb + warps < full;
+        const bool more = nxt < full;
+        const size_t nxt2 = more ? next_after(nxt) : full;
+        const T *px_next = x + nxt * kWarpElems + static_cast<size_t>(lane) * kLaneElems;   // read only if `more`
         uint32_t grp[4];
         if constexpr (kStages > 0) cp_async_wait<(kStages > 0 ? kStages - 1 : 0)>();   // the oldest stage has landed
 #pragma unroll
@@ -321,7 +338,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
                 o[e] = yv.x;
                 o[e + 1] = yv.y;
                 if constexpr (kIsBf16) {
-                    if (LUT && (e / 2) < Bf16LutPairs<BITS>::value) {              // resolved at compile time (unrolled)
+                    if constexpr (LUT) {
                         pc[e / 2] = lut[cell(cur[t], e)] + (static_cast<uint32_t>(lut[cell(cur[t], e + 1)]) << 16);
                     } else {
                         pc[e / 2] = bucketize_bf16x2<BITS, T>(prm.sb2, FOLD ? (pair_bits(cur[t], e) & 0x7fff7fffu) : pair_bits(cur[t], e));
@@ -364,7 +381,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
             }
         }
         if constexpr (kStages > 0) {                               // refill the stage just consumed
-            const size_t wbn = wb + kStages * warps;
+            const size_t wbn = kStages == 2 ? nxt2 : nxt;
             if (wbn < full) {
                 const T *px = x + wbn * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
 #pragma unroll
@@ -378,11 +395,15 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         uint32_t w[BITS];
         groups_to_words<BITS>(grp, w);
         store_words<BITS>(packed + wb * (32 * BITS) + (lane & 3) * (8 * BITS) + (lane >> 2) * BITS, w);
+        wb = nxt;
+        nxt = nxt2;
     }
 
     // ragged tail: the warp whose sequence reaches the index of the last, partial warp-block; a lane
     // owns 32 consecutive elements = BITS words
-    if ((n % kWarpElems) != 0 && all_full >= cta_begin && all_full < cta_end && (all_full - warp0) % warps == 0) {
+    const bool owns_tail = dynamic ? (blockIdx.x == 0 && threadIdx.x < 32)
+                                   : (all_full >= cta_begin && all_full < cta_end && (all_full - warp0) % warps == 0);
+    if ((n % kWarpElems) != 0 && owns_tail) {
         const size_t full = all_full;
         const size_t base = full * kWarpElems + static_cast<size_t>(lane) * 32;
         uint32_t w[BITS + 1];
@@ -501,8 +522,8 @@ struct FwdLaunchers { FwdLaunch fn[kMaxBits][3][2][2]; };
 template <int ACT, int BITS, bool FOLD>
 constexpr void fill_fwd_launchers(FwdLaunchers &l) {
     // 1-2 bit binary32 tables: the search is 1-3 comparisons, cheaper than the table;
-    // bfloat16: the table only where Bf16LutPairs says so
-    constexpr bool kLutF32 = BITS >= 3, kLutBf16 = Bf16LutPairs<BITS>::value > 0;
+    // 16-bit types: the packed search is 1-3 comparisons per element pair
+    constexpr bool kLutF32 = BITS >= 3, kLutBf16 = BITS >= 3;
     l.fn[BITS - 1][0][0][FOLD] = launch_fwd<ACT, BITS, float, false, FOLD>;
     l.fn[BITS - 1][0][1][FOLD] = launch_fwd<ACT, BITS, float, kLutF32, FOLD>;
     l.fn[BITS - 1][1][0][FOLD] = launch_fwd<ACT, BITS, __nv_bfloat16, false, FOLD>;

@@ -44,6 +44,29 @@ float f16_bits_to_float(uint32_t h);
 
 }  // namespace fewbit
 
+// ---- work counters of the dynamically scheduled forward variants (fewbit_queue.cu) ----------
+// A launch that distributes warp-blocks dynamically needs kQueues zeroed 32-bit counters,
+// kQueueStride words apart, that no other running kernel uses.  They live in a file-scope
+// __device__ pool of kQueueSlots sets; a set is leased per launch.
+#include <cuda_runtime_api.h>
+namespace fewbit {
+constexpr uint32_t kQueues = 16;
+constexpr uint32_t kQueueStride = 64;               // 32-bit words (256 bytes)
+constexpr int kQueueSlots = 16;
+
+struct QueueLease {
+    uint32_t *counters = nullptr;                   // device address; nullptr: no set free, use the static partition
+    int slot = -1;
+};
+// Picks a set that is safe to reuse (last used on this very stream, or by work that has completed),
+// and enqueues its clearing on `stream`.  Leaves the lease empty while `stream` is being captured
+// or when every set is still in use by other streams.
+cudaError_t queue_acquire(cudaStream_t stream, QueueLease *lease);
+// After the kernel launch (also after a failed one): records the point of `stream` up to which
+// the set is in use.
+cudaError_t queue_release(const QueueLease &lease, cudaStream_t stream);
+}  // namespace fewbit
+
 // The parameters s and y of Eq. 2, as binary32.  Unused boundary slots hold
 // +inf (never below any x), unused level slots 0.
 struct fewbit_table {

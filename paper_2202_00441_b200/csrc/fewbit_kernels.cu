@@ -154,28 +154,48 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
         prm.sb2[m] = dtype == FEWBIT_F16 ? table->s_f16x2[m] : table->s_bf16x2[m];
     }
     prm.runs = dtype == FEWBIT_F16 ? table->runs_f16 : (bf16 ? table->runs_bf16 : table->runs_f32);
+    prm.queue = nullptr;
     // the shared-memory code table pays off only when every warp of a one-wave grid gets enough work
     cudaError_t sm_err = cudaSuccess;
     const size_t slots = static_cast<size_t>(device_sm_count(&sm_err)) * (bf16 ? FwdCtas<__nv_bfloat16, true>::value : FwdCtas<float, true>::value);
     if (sm_err != cudaSuccess) { t_last_cuda_error = static_cast<int>(sm_err); return FEWBIT_ERR_CUDA; }
     const size_t warps_per_cta = static_cast<size_t>(bf16 ? FwdThreads<__nv_bfloat16, true>::value : FwdThreads<float, true>::value) / 32;
     const size_t waves = n / kWarpElems / (warps_per_cta * slots);
-    bool use_lut = prm.runs.count != 0 && waves >= kLutMinIters;
+    // 16-bit types (measured at 2^24 .. 2^28 elements, dynamic distribution): the table wins from ~6
+    // waves at 4 bits, from ~20 at 3 bits (the packed search costs 3 comparisons there, 4 levels of
+    // selects at 4 bits)
+    bool use_lut = prm.runs.count != 0 && ((table->bits == 4 && waves >= 6) || (table->bits == 3 && waves >= 20));
     if (!bf16 && prm.runs.count != 0) {
         // binary32 (measured, 2^22 .. 2^27 elements): at 4 bits the table beats the 4-level search at
         // every size; at 3 bits only on large inputs, and for the light activations never
         const int weight = act_weight(table->act);
         use_lut = table->bits == 4 || (table->bits == 3 && ((weight == 2 && waves >= kLutMinIters) || (weight == 1 && waves >= 24)));
     }
+    bool forced_table = false;
     if (const char *force = getenv("FEWBIT_FWD_TABLE")) {               // testing aid, see fewbit.h
-        if (force[0] == 'a') use_lut = prm.runs.count != 0;               // "always"
+        if (force[0] == 'a') { use_lut = prm.runs.count != 0; forced_table = true; }   // "always"
         else if (force[0] == 'n') use_lut = false;                        // "never"
     }
+    // 16-bit types: the table variant distributes its warp-blocks dynamically when a set of work
+    // counters can be leased (not during stream capture); at 3 bits it only beats the packed search
+    // that way
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    QueueLease lease;
+    const char *queue_mode = getenv("FEWBIT_FWD_QUEUE");               // testing aid: "never" keeps the static partition
+    if (use_lut && bf16 && !(queue_mode && queue_mode[0] == 'n')) {
+        const cudaError_t qerr = queue_acquire(st, &lease);
+        if (qerr != cudaSuccess) { t_last_cuda_error = static_cast<int>(qerr); return FEWBIT_ERR_CUDA; }
+        prm.queue = lease.counters;
+    }
+    if (use_lut && bf16 && table->bits == 3 && prm.queue == nullptr && !forced_table) use_lut = false;
     const FwdLaunch launch = fwd_launchers(table->act).fn[table->bits - 1][static_cast<int>(dtype)][use_lut][table->folded ? 1 : 0];
-    if (launch == nullptr) return FEWBIT_ERR_UNSUPPORTED;
-    const cudaError_t err = launch(
-        prm, x, y, packed, n, static_cast<cudaStream_t>(stream));
-    if (err != cudaSuccess) { t_last_cuda_error = static_cast<int>(err); return FEWBIT_ERR_CUDA; }
+    if (launch == nullptr) return FEWBIT_ERR_UNSUPPORTED;     // (no lease is held here: the table variants exist whenever runs.count != 0)
+    const cudaError_t err = launch(prm, x, y, packed, n, st);
+    const cudaError_t rerr = queue_release(lease, st);
+    if (err != cudaSuccess || rerr != cudaSuccess) {
+        t_last_cuda_error = static_cast<int>(err != cudaSuccess ? err : rerr);
+        return FEWBIT_ERR_CUDA;
+    }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return FEWBIT_OK;
 }

@@ -62,6 +62,7 @@ __device__ __forceinline__ float2 rcp_2(float2 a) { return make_float2(rcp_ftz(a
 template <int ACT>
 __device__ __forceinline__ float2 act_bf16(float2 x) {
     if constexpr (ACT == FEWBIT_GELU) {
+#if FEWBIT_GELU_BF16_RATIONAL
         // x Phi(x) = max(x,0) - t Phi(-t), t = |x|, and
         // t Phi(-t) = t e^{-t^2/2} G(w), w = 1/(1 + p t): G is a cubic times w fitted to
         // Phi(-t) e^{t^2/2} on [0, 14.5] with relative error 2.3e-4 (the fit is
@@ -75,6 +76,24 @@ __device__ __forceinline__ float2 act_bf16(float2 x) {
         g = fma2(g, w, splat(0.11820479f));
         const float2 q = mul2(mul2(g, w), e);
         return fma2(mul2(t, q), splat(-kScaleDown), relu);
+#else
+        // x Phi(x) = max(x,0) - t Phi(-t), t = |x|, and t Phi(-t) = 16 s 2^{L(s)} with
+        // s = min(t, 16) / 16 (one saturating multiply) and L(s) = log2 Phi(-16 s) a degree-8
+        // polynomial (fit_coefficients.py: relative error of the product 2.6e-4 up to t = 14.6, where
+        // it leaves the bfloat16 range; bounded beyond).  One ex2 per element and no reciprocal.
+        // The constant term carries log2(16) and the exponent offset S.
+        const float2 relu = relu2(x);
+        const float2 s = make_float2(__saturatef(fabsf(x.x) * 0.0625f), __saturatef(fabsf(x.y) * 0.0625f));
+        float2 l = fma2(s, splat(75.2134781f), splat(-330.892365f));
+        l = fma2(l, s, splat(623.153931f));
+        l = fma2(l, s, splat(-661.773987f));
+        l = fma2(l, s, splat(442.331207f));
+        l = fma2(l, s, splat(-199.337128f));
+        l = fma2(l, s, splat(-119.318939f));
+        l = fma2(l, s, splat(-18.3537769f));
+        l = fma2(l, s, splat(-1.00036657f + 4.0f + kScaleUp));
+        return fma2(mul2(s, ex2_2(l)), splat(-kScaleDown), relu);
+#endif
     } else if constexpr (ACT == FEWBIT_SILU) {
         // x sigmoid(x) = max(x,0) - |x| E / (1 + E)
         const float2 relu = relu2(x);

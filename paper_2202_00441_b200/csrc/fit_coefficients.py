@@ -12,6 +12,12 @@ build or run time.
 
    The binary16 kernel uses the same form with p = 0.38 and five terms.
 
+1b. GELU for bfloat16 storage, one exponential and no reciprocal.
+   t Phi(-t) = t 2^{L(t)},  L(t) = log2 Phi(-t), fitted by a polynomial in s = t / tmax on
+   s in [0, 1] (Chebyshev basis, absolute error of L minimised where t Phi(-t) is still
+   representable, loosely beyond); the kernel evaluates s = min(|x|, tmax) / tmax with a
+   saturating multiply.  bfloat16: tmax = 16, degree 8 (relative error of t Phi(-t) 2.6e-4).
+
 2. exp for binary32 storage.
    e^r = 1 + r + r^2 Q(r) on |r| <= ln(2)/2, Q of degree 4, relative error of
    e^r minimised the same way on Chebyshev nodes.
@@ -47,6 +53,26 @@ def fit_gelu_bf16(p=0.30, terms=4):
     return p * c, err          # coefficients of G(w) / w
 
 
+def fit_gelu_log2(tmax=16.0, deg=8, t_accurate=14.7, nodes=800):
+    from numpy.polynomial import chebyshev as C, polynomial as P
+    k = np.arange(nodes)
+    z = np.cos(np.pi * (k + 0.5) / nodes)
+    sv = (z + 1) / 2
+    target = np.array([float(mp.log(mp.ncdf(-mp.mpf(tmax * v)), 2)) for v in sv])
+    imp = np.where(tmax * sv <= t_accurate, 1.0, 0.02)
+    w = np.ones(nodes)
+    V = C.chebvander(z, deg)
+    for _ in range(60):
+        c, *_ = np.linalg.lstsq(V * (w * imp)[:, None], target * w * imp, rcond=None)
+        err = (V @ c - target) * imp
+        w = w * (1 + 4 * np.abs(err) / np.abs(err).max())
+        w /= w.mean()
+    mono = np.zeros(1)
+    for cf in C.cheb2poly(c)[::-1]:
+        mono = P.polyadd(P.polymul(mono, [-1.0, 2.0]), [cf])       # z = 2 s - 1
+    return mono, np.abs(err).max()
+
+
 def fit_exp_f32(deg_q=4):
     half = float(mp.log(2) / 2) * 1.0005
     k = np.arange(400)
@@ -77,6 +103,9 @@ if __name__ == "__main__":
     c, err = fit_gelu_bf16()
     print("GELU bf16: p = 0.30, G(w)/w coefficients (c0..c3):", [float(np.float32(v)) for v in c],
           "max relative error %.3e" % err)
+    c, err = fit_gelu_log2()
+    print("GELU bf16 (log2 form): L(16 s) coefficients (s^0..s^8):", ", ".join("%.9g" % np.float32(v) for v in c),
+          "max error of L %.3e" % err)
     c, err = fit_gelu_bf16(p=0.38, terms=5)
     print("GELU f16: p = 0.38, G(w)/w coefficients (c0..c4):", [float(v) for v in c], "max relative error %.3e" % err)
     g, err = fit_gelu_f32()

@@ -380,6 +380,55 @@ def test_runs_on_a_side_stream():
     compare_full("silu", 4, x, g, y, p, gi, "side stream")
 
 
+@pytest.mark.parametrize("bits", [3, 4])
+def test_dynamic_table_variant_on_concurrent_streams(bits, monkeypatch):
+    """The table variant of the 16-bit types hands out warp-blocks through leased work counters.
+    Three streams at once, twice each (a stream reuses its own counters, different streams must
+    not share any): every launch gives exactly what the search variant gives on the same input,
+    and that agrees with the oracle on sampled blocks."""
+    n = (1 << 25) + 4097
+    t = table("gelu", bits)
+    gen = torch.Generator(device=DEV).manual_seed(31 + bits)
+    xs = [torch.randn(n, device=DEV, generator=gen).bfloat16() for _ in range(3)]
+    monkeypatch.setenv("FEWBIT_FWD_TABLE", "never")
+    refs = [fb.fewbit_fwd(t, x) for x in xs]
+    torch.cuda.synchronize()
+    g = torch.ones(n, device=DEV).bfloat16()
+    compare_sampled("gelu", bits, xs[0], g, refs[0][0], refs[0][1], fb.fewbit_bwd(t, refs[0][1], g), "search variant")
+    monkeypatch.setenv("FEWBIT_FWD_TABLE", "always")
+    streams = [torch.cuda.Stream() for _ in xs]
+    outs = []
+    for rep in range(2):
+        for x, st in zip(xs, streams):
+            st.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(st):
+                outs.append(fb.fewbit_fwd(t, x))
+    for st in streams:
+        st.synchronize()
+    for i, (y, pk) in enumerate(outs):
+        y_ref, p_ref = refs[i % 3]
+        assert torch.equal(pk, p_ref), f"codes differ, launch {i}"
+        assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16)), f"y differs, launch {i}"
+
+
+def test_stream_capture_uses_the_static_partition_and_replays():
+    """No work counters are leased while a stream is being captured; the captured launch gives the
+    same result as the eager (dynamically distributed) one."""
+    n = 1 << 25
+    t = table("silu", 4)
+    x = torch.randn(n, device=DEV).bfloat16()
+    y, pk = fb.fewbit_fwd(t, x)                     # eager: also resolves every per-device one-time setting
+    torch.cuda.synchronize()
+    y2, p2 = torch.zeros_like(y), torch.zeros_like(pk)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        fb.fewbit_fwd(t, x, y2, p2)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(p2, pk)
+    assert torch.equal(y2.view(torch.int16), y.view(torch.int16))
+
+
 # --------------------------------------------------------------------------
 # host-buffer entry points
 # --------------------------------------------------------------------------
