@@ -176,13 +176,14 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
         if (force[0] == 'a') { use_lut = prm.runs.count != 0; forced_table = true; }   // "always"
         else if (force[0] == 'n') use_lut = false;                        // "never"
     }
-    // 16-bit types: the table variant distributes its warp-blocks dynamically when a set of work
-    // counters can be leased (not during stream capture); at 3 bits it only beats the packed search
-    // that way
+    // The table variants distribute their warp-blocks dynamically when a set of work counters can
+    // be leased (not during stream capture); the 16-bit types at 3 bits only beat the packed search
+    // that way.  binary32 ReLU / leaky ReLU measured faster with short CTAs and a static partition,
+    // and below two waves there is nothing to balance.
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     QueueLease lease;
     const char *queue_mode = getenv("FEWBIT_FWD_QUEUE");               // testing aid: "never" keeps the static partition
-    if (use_lut && bf16 && !(queue_mode && queue_mode[0] == 'n')) {
+    if (use_lut && (bf16 || (act_weight(table->act) >= 1 && waves >= 2)) && !(queue_mode && queue_mode[0] == 'n')) {
         const cudaError_t qerr = queue_acquire(st, &lease);
         if (qerr != cudaSuccess) { t_last_cuda_error = static_cast<int>(qerr); return FEWBIT_ERR_CUDA; }
         prm.queue = lease.counters;

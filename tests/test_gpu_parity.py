@@ -411,6 +411,25 @@ def test_dynamic_table_variant_on_concurrent_streams(bits, monkeypatch):
         assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16)), f"y differs, launch {i}"
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_dynamic_and_static_partition_agree_on_whole_arrays(dtype, monkeypatch):
+    """Every element and every packed word of the dynamically distributed table variant equals the
+    statically partitioned one (a warp-block dropped or done twice would show), ragged tail included."""
+    n = (1 << 24) + 4097
+    x = (torch.randn(n, device=DEV) * 2).to(TORCH_DT[dtype])
+    monkeypatch.setenv("FEWBIT_FWD_TABLE", "always")
+    for act in ("sigmoid", "gelu"):
+        for bits in (3, 4):
+            t = table(act, bits)
+            monkeypatch.setenv("FEWBIT_FWD_QUEUE", "never")
+            y0, p0 = fb.fewbit_fwd(t, x)
+            monkeypatch.delenv("FEWBIT_FWD_QUEUE")
+            y1, p1 = fb.fewbit_fwd(t, x)
+            torch.cuda.synchronize()
+            assert torch.equal(p0, p1), (dtype, act, bits)
+            assert torch.equal(y0.view(torch.uint8), y1.view(torch.uint8)), (dtype, act, bits)
+
+
 def test_stream_capture_uses_the_static_partition_and_replays():
     """No work counters are leased while a stream is being captured; the captured launch gives the
     same result as the eager (dynamically distributed) one."""
