@@ -16,7 +16,7 @@
 //                      2^-64 is folded into the last fused multiply-add, whose
 //                      IEEE gradual underflow gives correct subnormals.
 //   T = half     : as bfloat16 where the hardware approximation is 2^-22 (ex2, rcp, lg2), with a
-//                  longer GELU fit (3.5e-5) and tanh / expm1 from ex2 instead of tanh.approx
+//                  tighter GELU fit (3.4e-5) and tanh / expm1 from ex2 instead of tanh.approx
 //                  (2^-11 is not enough for 11 significant bits).
 //   T = float    : binary32 arithmetic built on an exponential good to ~0.7 ulp, with the
 //                  rounding error of every step that would reach the result carried along as a
@@ -62,21 +62,6 @@ __device__ __forceinline__ float2 rcp_2(float2 a) { return make_float2(rcp_ftz(a
 template <int ACT>
 __device__ __forceinline__ float2 act_bf16(float2 x) {
     if constexpr (ACT == FEWBIT_GELU) {
-#if FEWBIT_GELU_BF16_RATIONAL
-        // x Phi(x) = max(x,0) - t Phi(-t), t = |x|, and
-        // t Phi(-t) = t e^{-t^2/2} G(w), w = 1/(1 + p t): G is a cubic times w fitted to
-        // Phi(-t) e^{t^2/2} on [0, 14.5] with relative error 2.3e-4 (the fit is
-        // paper_2202_00441_b200/csrc/fit_coefficients.py)
-        const float2 relu = relu2(x);
-        const float2 t = abs2_from_relu(relu, x);
-        const float2 e = ex2_2(fma2(mul2(x, x), splat(-0.5f * kLog2e), splat(kScaleUp)));
-        const float2 w = rcp_2(fma2(t, splat(0.30f), splat(1.0f)));
-        float2 g = fma2(w, splat(0.20884148f), splat(0.03559305f));
-        g = fma2(g, w, splat(0.13747554f));
-        g = fma2(g, w, splat(0.11820479f));
-        const float2 q = mul2(mul2(g, w), e);
-        return fma2(mul2(t, q), splat(-kScaleDown), relu);
-#else
         // x Phi(x) = max(x,0) - t Phi(-t), t = |x|, and t Phi(-t) = 16 s 2^{L(s)} with
         // s = min(t, 16) / 16 (one saturating multiply) and L(s) = log2 Phi(-16 s) a degree-8
         // polynomial (fit_coefficients.py: relative error of the product 2.6e-4 up to t = 14.6, where
@@ -93,7 +78,6 @@ __device__ __forceinline__ float2 act_bf16(float2 x) {
         l = fma2(l, s, splat(-18.3537769f));
         l = fma2(l, s, splat(-1.00036657f + 4.0f + kScaleUp));
         return fma2(mul2(s, ex2_2(l)), splat(-kScaleDown), relu);
-#endif
     } else if constexpr (ACT == FEWBIT_SILU) {
         // x sigmoid(x) = max(x,0) - |x| E / (1 + E)
         const float2 relu = relu2(x);
@@ -343,17 +327,18 @@ __device__ __forceinline__ float2 act_f32(float2 x) {
 template <int ACT>
 __device__ __forceinline__ float2 act_f16(float2 x) {
     if constexpr (ACT == FEWBIT_GELU) {
-        // as for bfloat16, with a 5-term fit (p = 0.38, relative error 3.5e-5; fit_coefficients.py)
+        // as for bfloat16: t Phi(-t) = 6 s 2^{L(s)}, s = min(t, 6) / 6, L(s) = log2 Phi(-6 s) of degree 6
+        // (relative error of the product 3.4e-5 up to t = 5.7; beyond, the product is below half the
+        // smallest binary16 subnormal and stays there: 6 * 2^L(1) = 6e-9)
         const float2 relu = relu2(x);
-        const float2 t = abs2_from_relu(relu, x);
-        const float2 e = ex2_2(fma2(mul2(x, x), splat(-0.5f * kLog2e), splat(kScaleUp)));
-        const float2 w = rcp_2(fma2(t, splat(0.38f), splat(1.0f)));
-        float2 g = fma2(w, splat(-0.08992644399404526f), splat(0.1888723224401474f));
-        g = fma2(g, w, splat(0.09198290854692459f));
-        g = fma2(g, w, splat(0.15782848000526428f));
-        g = fma2(g, w, splat(0.1512252390384674f));
-        const float2 q = mul2(mul2(g, w), e);
-        return fma2(mul2(t, q), splat(-kScaleDown), relu);
+        const float2 s = make_float2(__saturatef(fabsf(x.x) * 0.16666667f), __saturatef(fabsf(x.y) * 0.16666667f));
+        float2 l = fma2(s, splat(1.16089976f), splat(-4.98774767f));
+        l = fma2(l, s, splat(9.55984306f));
+        l = fma2(l, s, splat(-11.1624165f));
+        l = fma2(l, s, splat(-16.5841904f));
+        l = fma2(l, s, splat(-6.90263224f));
+        l = fma2(l, s, splat(-1.00004601f + 2.5849625f + kScaleUp));
+        return fma2(mul2(s, ex2_2(l)), splat(-kScaleDown), relu);
     } else if constexpr (ACT == FEWBIT_TANH) {
         // |x| >= 1/32: (1 - E) / (1 + E), E = e^{-2|x|} (1 - E >= 0.06, no harmful cancellation);
         // below: x - x^3/3 (relative error 2 x^4 / 15 < 2e-7)

@@ -3,20 +3,15 @@
 Run by hand (needs numpy and mpmath); prints the constants.  Not used at
 build or run time.
 
-1. GELU for bfloat16 storage.
+1. GELU for bfloat16 and binary16 storage, one exponential and no reciprocal.
    x Phi(x) = max(x,0) - t Phi(-t), t = |x|, and
-   t Phi(-t) = t exp(-t^2/2) G(w),  w = 1/(1 + p t),  G(w) = p w (c0 + c1 w + c2 w^2 + c3 w^3).
-   Fit of (1 - w) (c0 + ... + c3 w^3) to t Phi(-t) exp(t^2/2) on t in (0, 14.5]
-   (note (1 - w) = p t w), relative error minimised by iteratively reweighted
-   least squares.  The kernel needs ~2^-10 relative accuracy.
-
-   The binary16 kernel uses the same form with p = 0.38 and five terms.
-
-1b. GELU for bfloat16 storage, one exponential and no reciprocal.
    t Phi(-t) = t 2^{L(t)},  L(t) = log2 Phi(-t), fitted by a polynomial in s = t / tmax on
    s in [0, 1] (Chebyshev basis, absolute error of L minimised where t Phi(-t) is still
-   representable, loosely beyond); the kernel evaluates s = min(|x|, tmax) / tmax with a
-   saturating multiply.  bfloat16: tmax = 16, degree 8 (relative error of t Phi(-t) 2.6e-4).
+   representable in the storage type, loosely beyond); the kernel evaluates
+   s = min(|x|, tmax) / tmax with a saturating multiply.
+   bfloat16: tmax = 16, degree 8, accurate up to t = 14.7 (relative error of t Phi(-t) 2.6e-4).
+   binary16: tmax = 6, degree 6, accurate up to t = 5.7 (3.4e-5); beyond, t Phi(-t) is below
+   half the smallest subnormal.
 
 2. exp for binary32 storage.
    e^r = 1 + r + r^2 Q(r) on |r| <= ln(2)/2, Q of degree 4, relative error of
@@ -42,15 +37,6 @@ def minimax_lstsq(A, target, weight_of_error, iters=60):
         w = w * (1 + 4 * np.abs(err) / np.abs(err).max())
         w /= w.mean()
     return c, np.abs(err).max()
-
-
-def fit_gelu_bf16(p=0.30, terms=4):
-    ts = np.concatenate([np.linspace(1e-4, 1, 400), np.linspace(1, 14.5, 1200)])
-    tq = np.array([float(mp.mpf(t) * mp.ncdf(-mp.mpf(t)) * mp.exp(mp.mpf(t) ** 2 / 2)) for t in ts])
-    w = 1 / (1 + p * ts)
-    A = np.stack([(1 - w) * w ** i for i in range(terms)], 1)
-    c, err = minimax_lstsq(A / tq[:, None], np.ones_like(tq), lambda e: e)
-    return p * c, err          # coefficients of G(w) / w
 
 
 def fit_gelu_log2(tmax=16.0, deg=8, t_accurate=14.7, nodes=800):
@@ -100,14 +86,12 @@ def fit_gelu_f32(p=0.2, deg=9, centre=0.5, tmax=15.0, nodes=500):
 
 
 if __name__ == "__main__":
-    c, err = fit_gelu_bf16()
-    print("GELU bf16: p = 0.30, G(w)/w coefficients (c0..c3):", [float(np.float32(v)) for v in c],
-          "max relative error %.3e" % err)
     c, err = fit_gelu_log2()
-    print("GELU bf16 (log2 form): L(16 s) coefficients (s^0..s^8):", ", ".join("%.9g" % np.float32(v) for v in c),
+    print("GELU bf16: L(16 s) coefficients (s^0..s^8):", ", ".join("%.9g" % np.float32(v) for v in c),
           "max error of L %.3e" % err)
-    c, err = fit_gelu_bf16(p=0.38, terms=5)
-    print("GELU f16: p = 0.38, G(w)/w coefficients (c0..c4):", [float(v) for v in c], "max relative error %.3e" % err)
+    c, err = fit_gelu_log2(tmax=6.0, deg=6, t_accurate=5.7)
+    print("GELU f16: L(6 s) coefficients (s^0..s^6):", ", ".join("%.9g" % np.float32(v) for v in c),
+          "max error of L %.3e" % err)
     g, err = fit_gelu_f32()
     c0 = np.float32(g[0])
     print("GELU f32: p = float32(0.2), G in u = w - 1/2: c0 = %.9g + %.9g, c1..c9 =" % (c0, np.float32(g[0] - float(c0))),
