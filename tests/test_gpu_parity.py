@@ -96,12 +96,12 @@ def compare_full(act, bits, x, g, y, packed, gi, what):
     compare_block(act, bits, np_bits(x), np_bits(g), np_bits(y), np_bits(packed).view(np.uint32), np_bits(gi), what)
 
 
-def compare_sampled(act, bits, x, g, y, packed, gi, what, blocks=24, block_elems=8192, seed=0):
+def compare_sampled(act, bits, x, g, y, packed, gi, what, blocks=24, block_elems=8192, seed=0, also_at=()):
     """Element-by-element comparison on randomly placed 32-aligned blocks plus
-    the first and the last (ragged) block."""
+    the first and the last (ragged) block (and blocks starting at `also_at`)."""
     n = x.numel()
     rng = np.random.default_rng(seed)
-    starts = {0, max(0, (n - block_elems) // 32 * 32)}
+    starts = {0, max(0, (n - block_elems) // 32 * 32)} | {int(a) // 32 * 32 for a in also_at}
     while len(starts) < blocks:
         starts.add(int(rng.integers(0, max(1, n - block_elems))) // 32 * 32)
     jobs = []
@@ -187,6 +187,30 @@ def test_config5_sweep_large_sampled(n, dtype):
             compare_sampled(act, bits, x, g, y, p, gi, f"c5 {act} k={bits} n={n} {dtype}", blocks=blocks,
                             block_elems=4096, seed=bits)
             del y, p, gi
+
+
+def test_more_than_2_to_the_32_elements():
+    """Element and word indices beyond 32 bits: 2^32 + 3149 bfloat16 elements (about 28 GB on the
+    device), 1 bit (search variant) and 4 bits (table variant, dynamically distributed); sampled
+    blocks include the ones that straddle element 2^32 and the ragged tail."""
+    n = (1 << 32) + 3 * 1024 + 77
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2 ** 30:
+        pytest.skip("needs ~28 GB of free device memory")
+    x = torch.empty(n, device=DEV, dtype=torch.bfloat16)
+    gen = torch.Generator(device=DEV).manual_seed(5)
+    step = 1 << 28
+    for e0 in range(0, n, step):
+        m = min(step, n - e0)
+        x[e0:e0 + m] = torch.randn(m, device=DEV, generator=gen).mul_(1.5).bfloat16()
+    near = [(1 << 32) - 4096, (1 << 32) - 32, 1 << 32, (1 << 31) - 4096, 1 << 31]
+    for bits in (1, 4):
+        t = table("silu", bits)
+        y, pk = fb.fewbit_fwd(t, x)
+        gi = fb.fewbit_bwd(t, pk, x)                # the input doubles as the incoming gradient
+        torch.cuda.synchronize()
+        compare_sampled("silu", bits, x, x, y, pk, gi, f"2^32+ k={bits}", blocks=16, seed=bits, also_at=near)
+        del y, pk, gi
 
 
 # --------------------------------------------------------------------------
