@@ -190,7 +190,7 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  * through a set of counters in a
  * file-scope device array (16 sets per device; nothing is allocated, but the
  * first such call on a device creates up to 16 CUDA events, and each call
- * enqueues a 4 KB clear ahead of the kernel).  While `stream` is being captured,
+ * records one after its kernel).  While `stream` is being captured,
  * or when all sets are in use by other streams, the kernel falls back to a
  * static partition: same results, ~10 % slower.  Environment variables for
  * testing and tuning only: FEWBIT_FWD_TABLE = always | never | auto (use of

@@ -426,6 +426,23 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         for (int j = 0; j < BITS; ++j)
             if (first + j < total_words) packed[first + j] = w[j];
     }
+
+    // Dynamic distribution: the last CTA of the grid to get here puts the work counters back to
+    // zero for the next launch that leases them (every warp has made its last claim by then).
+    if constexpr (LUT) {
+        if (dynamic) {                                              // uniform over the grid
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                __threadfence();
+                if (atomicAdd(prm.queue + kQueueDoneWord, 1u) == gridDim.x - 1) {
+#pragma unroll
+                    for (uint32_t q = 0; q < kQueues; ++q) prm.queue[q * kQueueStride] = 0;
+                    prm.queue[kQueueDoneWord] = 0;
+                    __threadfence();
+                }
+            }
+        }
+    }
 }
 
 template <typename T, bool LUT>

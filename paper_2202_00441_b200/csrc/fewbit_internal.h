@@ -47,20 +47,22 @@ float f16_bits_to_float(uint32_t h);
 // ---- work counters of the dynamically scheduled forward variants (fewbit_queue.cu) ----------
 // A launch that distributes warp-blocks dynamically needs kQueues zeroed 32-bit counters,
 // kQueueStride words apart, that no other running kernel uses.  They live in a file-scope
-// __device__ pool of kQueueSlots sets; a set is leased per launch.
+// __device__ pool of kQueueSlots sets (zero-initialised); a set is leased per launch and the
+// kernel itself puts it back to zero when its last CTA finishes.
 #include <cuda_runtime_api.h>
 namespace fewbit {
 constexpr uint32_t kQueues = 16;
 constexpr uint32_t kQueueStride = 64;               // 32-bit words (256 bytes)
 constexpr int kQueueSlots = 16;
+constexpr uint32_t kQueueDoneWord = kQueueStride / 2;   // in the padding behind counter 0: CTAs that have finished
 
 struct QueueLease {
     uint32_t *counters = nullptr;                   // device address; nullptr: no set free, use the static partition
     int slot = -1;
 };
-// Picks a set that is safe to reuse (last used on this very stream, or by work that has completed),
-// and enqueues its clearing on `stream`.  Leaves the lease empty while `stream` is being captured
-// or when every set is still in use by other streams.
+// Picks a set that is safe to reuse (last used on this very stream, or by work that has completed).
+// Leaves the lease empty while `stream` is being captured or when every set is still in use by
+// other streams.
 cudaError_t queue_acquire(cudaStream_t stream, QueueLease *lease);
 // After the kernel launch (also after a failed one): records the point of `stream` up to which
 // the set is in use.

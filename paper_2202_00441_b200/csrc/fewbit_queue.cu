@@ -4,8 +4,9 @@
 // is resolved once per device with cudaGetSymbolAddress).  What is created lazily is one CUDA event
 // per set and device, used to learn whether the last kernel that used the set has finished.
 // A set is handed out again
-//   * to the stream that used it last without any wait (stream order puts the clearing after the
-//     previous kernel; streams are told apart by cudaStreamGetId, which is never reused), or
+//   * to the stream that used it last without any wait (stream order puts the new kernel after the
+//     previous one, whose last CTA has zeroed the counters; streams are told apart by
+//     cudaStreamGetId, which is never reused), or
 //   * to any stream once its event has completed.
 // While a stream is being captured no set is leased (an event query is not allowed there): the
 // caller then uses the static partition.
@@ -78,9 +79,7 @@ cudaError_t queue_acquire(cudaStream_t stream, QueueLease *lease) {
         err = cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming);
         if (err != cudaSuccess) { s.done = nullptr; return err; }
     }
-    uint32_t *set = st.base + static_cast<size_t>(pick) * kSetWords;
-    err = cudaMemsetAsync(set, 0, kSetWords * sizeof(uint32_t), stream);
-    if (err != cudaSuccess) return err;
+    uint32_t *set = st.base + static_cast<size_t>(pick) * kSetWords;     // all zero: never used, or reset by its last kernel
     s.leased = true;
     s.stream_id = id;
     lease->counters = set;
