@@ -135,7 +135,6 @@ __device__ __forceinline__ void load_raw_shared(uint32_t saddr, Raw<float> &r) {
 
 struct FwdSmem {
     uint32_t runs[kMaxRuns + 1];     // start | value << 24, plus a sentinel run starting one past the last cell
-    uint32_t work[kMaxRuns + 1];     // [0] = count, then 16-cell groups that straddle a run boundary
     float thr[kMaxLevels];           // the boundaries, for the binary32 one-comparison step
 };
 
@@ -154,10 +153,11 @@ template <int CELLS, int THREADS>
 __device__ __forceinline__ void expand_runs(const CodeRuns &enc, uint8_t *lut, FwdSmem &sm) {
     const uint32_t count = enc.count;
     for (uint32_t i = threadIdx.x; i <= count; i += THREADS) sm.runs[i] = (i < count) ? enc.run[i] : static_cast<uint32_t>(CELLS);
-    if (threadIdx.x == 0) sm.work[0] = 0;
     __syncthreads();
     // A warp owns a contiguous stretch of 16-cell groups; lane l takes groups l, l + 32, ... of it,
     // so that the 128-bit stores of one instruction fall on consecutive addresses (no bank conflict).
+    // A group inside one run is one splat store; the few groups that straddle a run boundary (at
+    // most one per run) are assembled byte by byte in registers by the same thread.
     constexpr int kGroups = CELLS / 16;             // 16 cells = one 128-bit shared store
     constexpr int kWarps = THREADS / 32;
     constexpr int kPerWarp = (kGroups + kWarps - 1) / kWarps;
@@ -170,20 +170,22 @@ __device__ __forceinline__ void expand_runs(const CodeRuns &enc, uint8_t *lut, F
             const uint32_t g = first + 32 * i;
             if (g >= kGroups || g >= ((threadIdx.x >> 5) + 1) * kPerWarp) break;
             const uint32_t a = g * 16;
-            while ((sm.runs[r + 1] & 0xffffffu) <= a) ++r;
-            if ((sm.runs[r + 1] & 0xffffffu) >= a + 16) {
-                const uint32_t v = (sm.runs[r] >> 24) * 0x01010101u;
-                *reinterpret_cast<uint4 *>(lut + a) = make_uint4(v, v, v, v);
+            uint32_t next = sm.runs[r + 1] & 0xffffffu;
+            while (next <= a) { ++r; next = sm.runs[r + 1] & 0xffffffu; }
+            uint32_t w[4];
+            if (next >= a + 16) {
+                w[0] = w[1] = w[2] = w[3] = (sm.runs[r] >> 24) * 0x01010101u;
             } else {
-                sm.work[1 + atomicAdd(&sm.work[0], 1u)] = g;      // at most one group per run start
+                uint32_t rr = r, nn = next, v = sm.runs[r] >> 24;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    while (nn <= a + c) { ++rr; nn = sm.runs[rr + 1] & 0xffffffu; v = sm.runs[rr] >> 24; }
+                    if ((c & 3) == 0) w[c >> 2] = 0;
+                    w[c >> 2] |= v << (8 * (c & 3));
+                }
             }
+            *reinterpret_cast<uint4 *>(lut + a) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-    }
-    __syncthreads();
-    const uint32_t todo = sm.work[0] * 16;
-    for (uint32_t i = threadIdx.x; i < todo; i += THREADS) {
-        const uint32_t c = sm.work[1 + (i >> 4)] * 16 + (i & 15);
-        lut[c] = static_cast<uint8_t>(sm.runs[find_run(sm.runs, count, c)] >> 24);
     }
     __syncthreads();
 }
