@@ -197,6 +197,11 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  * the code-table variant, default auto), FEWBIT_FWD_QUEUE = never (static
  * partition), FEWBIT_FWD_ITERS = <k> (warp-blocks per warp) and
  * FEWBIT_FWD_WARPS = <w> (warps per CTA of the variants without a code table).
+ * Both device kernels are launched with programmatic stream serialization:
+ * their CTAs may be scheduled while the previous kernel of `stream` drains,
+ * and wait there for its completion before they touch memory, so stream order
+ * holds as usual (FEWBIT_PDL=0 in the environment launches them the ordinary
+ * way).
  */
 FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y,
                                     uint32_t *packed, size_t n, fewbit_dtype dtype, void *stream);

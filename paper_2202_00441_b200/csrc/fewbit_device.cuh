@@ -37,6 +37,30 @@ constexpr int kThreads = 256;
 constexpr int kWarpsPerCta = kThreads / 32;
 
 // ---------------------------------------------------------------------------
+// programmatic dependent launch: the next kernel of the stream may be scheduled once every CTA of
+// this grid has started; a kernel launched that way must not touch global memory before pdl_wait(),
+// which returns when the grids it depends on have completed and their writes are visible.  Both
+// are no-ops for a kernel launched the ordinary way.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... Params, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, bool pdl, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
+// ---------------------------------------------------------------------------
 // global memory access: 8 elements per lane, widened to binary32
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ void load8(const float *p, float (&v)[8]) {

@@ -244,6 +244,8 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
 template <int ACT, int BITS, typename T, bool LUT, bool FOLD>
 __global__ void __launch_bounds__(FwdThreads<T, LUT>::value, FwdCtas<T, LUT>::value)
 fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters) {
+    pdl_launch_dependents();
+    pdl_wait();
     constexpr bool kIsBf16 = sizeof(T) == 2;
     constexpr int kFwdThreads = FwdThreads<T, LUT>::value;
     constexpr int kCells = kIsBf16 ? (1 << kCellBitsBf16) : (1 << kCellBitsF32);
@@ -464,6 +466,7 @@ constexpr int act_weight(int act) {
 }
 constexpr size_t kLutMinIters = 8;      // below this many warp-blocks per warp the table does not pay for its expansion
 const char *fwd_iters_override();        // tuning aid: environment FEWBIT_FWD_ITERS
+bool pdl_enabled();
 const char *fwd_warps_override();        // tuning aid: environment FEWBIT_FWD_WARPS (variant without a table)
 
 template <int ACT, int BITS, typename T, bool LUT, bool FOLD>
@@ -531,9 +534,13 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     if (const char *dbg = fwd_iters_override()) iters = static_cast<size_t>(atoi(dbg));
     const size_t per_cta = warps_per_cta * iters;
     const unsigned grid = static_cast<unsigned>((warp_blocks + per_cta - 1) / per_cta);
-    kernel<<<grid, static_cast<unsigned>(warps_per_cta * 32), smem * warps_per_cta / (kFwdThreads / 32), st>>>(prm, static_cast<const T *>(x), static_cast<T *>(y), packed, n,
-                                             static_cast<int>(iters));
-    return cudaGetLastError();
+    // Programmatic dependent launch lets this grid's CTAs take their places while the previous kernel
+    // of the stream drains (they wait there for it to complete).  Not below one CTA per SM: the
+    // early CTAs land on the SMs the previous kernel left idle, two per SM, and an issue-bound
+    // sub-wave grid then runs on half the SMs (binary32 GELU, 2^20 elements: 8.3 -> 9.2 us).
+    const bool pdl = pdl_enabled() && grid >= static_cast<unsigned>(sms);
+    return launch_pdl(kernel, grid, static_cast<unsigned>(warps_per_cta * 32), smem * warps_per_cta / (kFwdThreads / 32), st, pdl,
+                      prm, static_cast<const T *>(x), static_cast<T *>(y), packed, n, static_cast<int>(iters));
 }
 
 using FwdLaunch = cudaError_t (*)(const FwdParams &, const void *, void *, uint32_t *, size_t, cudaStream_t);

@@ -15,9 +15,11 @@ thread_local int t_last_cuda_error = 0;
 template <int BITS, typename T>
 __global__ void __launch_bounds__(kThreads)
 bwd_kernel(const __grid_constant__ Levels tl, const uint32_t *packed, const T *grad_out, T *grad_in, size_t n) {
+    pdl_launch_dependents();
     __shared__ float lev[kMaxLevels];
     if (threadIdx.x < kMaxLevels) lev[threadIdx.x] = tl.lev[threadIdx.x];
     __syncthreads();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const size_t wb = static_cast<size_t>(blockIdx.x) * kWarpsPerCta + (threadIdx.x >> 5);
     const size_t full = n / kWarpElems;
@@ -71,8 +73,7 @@ inline unsigned bwd_grid_for(size_t n) {
 
 template <int BITS, typename T>
 cudaError_t launch_bwd(const Levels &tl, const uint32_t *packed, const void *g, void *gi, size_t n, cudaStream_t st) {
-    bwd_kernel<BITS, T><<<bwd_grid_for(n), kThreads, 0, st>>>(tl, packed, static_cast<const T *>(g), static_cast<T *>(gi), n);
-    return cudaGetLastError();
+    return launch_pdl(bwd_kernel<BITS, T>, bwd_grid_for(n), kThreads, 0, st, pdl_enabled(), tl, packed, static_cast<const T *>(g), static_cast<T *>(gi), n);
 }
 
 const BwdLaunch kBwd[kMaxBits][3] = {      // [bits - 1][dtype: f32, bf16, f16]
@@ -127,6 +128,11 @@ int device_sm_count(cudaError_t *err) {
 const char *fwd_iters_override() {
     static const char *v = getenv("FEWBIT_FWD_ITERS");
     return (v && *v) ? v : nullptr;
+}
+
+bool pdl_enabled() {
+    static const bool on = [] { const char *v = getenv("FEWBIT_PDL"); return !(v && v[0] == '0'); }();   // testing aid: FEWBIT_PDL=0
+    return on;
 }
 
 const char *fwd_warps_override() {
