@@ -1,22 +1,27 @@
 // Forward half of Listing 1 for sm_100a: y = f(x), code = position of x among
 // the boundaries (Eq. 2), codes bit-packed into whole 32-bit words.
 //
-// A CTA of 512 threads owns a contiguous stretch of 16 * iters warp-blocks of
-// 1024 elements; warp w takes warp-blocks w, w + 16, ... of it (see
-// fewbit_device.cuh for the lane / tile / warp-block decomposition and the quad
-// transpose that turns per-lane code groups into whole words).  The hardware
-// block scheduler balances the CTAs over the SMs (two resident per SM).
+// A warp works on warp-blocks of 1024 elements (see fewbit_device.cuh for the
+// lane / tile / warp-block decomposition and the quad transpose that turns
+// per-lane code groups into whole words).  Which warp-blocks a warp gets:
+//   * variants without a code table: a CTA owns a contiguous stretch of
+//     warps * iters warp-blocks, warp w takes w, w + warps, ... of it; the CTA
+//     size is chosen at launch (16-bit types: 4 warps) and the hardware block
+//     scheduler balances the CTAs over the SMs;
+//   * code-table variants: one wave of long-lived CTAs (the table is expanded
+//     once per CTA); the warp-blocks are handed out dynamically through leased
+//     work counters when a lease is available (fewbit_queue.cu), else statically
+//     as above.
 //
-// Bucketize (code = #{ j : s[j] < x }, Eq. 2) has three implementations, mixed
-// so that no single pipe of the SM saturates before HBM does:
+// Bucketize (code = #{ j : s[j] < x }, Eq. 2) has three implementations:
 //   search   : branch-free binary search on one binary32 element (ALU pipe);
-//   packed   : bfloat16 only -- the same search on TWO elements per
-//              instruction with bf16x2 compares against boundaries rounded
-//              down to bfloat16 (exact: s < x <=> floor_bf16(s) < x for a
-//              bfloat16 x), threshold selection by bitwise masks;
+//   packed   : 16-bit types -- the same search on TWO elements per
+//              instruction with bf16x2 / f16x2 compares against boundaries
+//              rounded down to the storage type (exact: s < x <=> floor(s) < x
+//              for an x of that type), threshold selection by bitwise masks;
 //   look-up  : the code is a step function of x, so it is read from a byte
 //              table in shared memory indexed by the top bits of the pattern:
-//                bfloat16 : 65 536 entries, one per pattern, the exact code;
+//                16-bit   : 65 536 entries, one per pattern, the exact code;
 //                binary32 : 8 192 entries (sign, exponent, 4 mantissa bits);
 //                           an entry m is the smallest code in its cell and
 //                           code = m + (s[m] < x), one binary32 comparison; a
@@ -26,9 +31,10 @@
 //              The table arrives run-length encoded as a kernel parameter (a
 //              few dozen runs) and is expanded by the CTA before streaming.
 //              Random indices cost ~3.3 shared-memory wavefronts per warp
-//              look-up, which is why bfloat16 uses it for only half of the
-//              elements and only at 4 bits.
-// LUT = false: no table (bfloat16: packed search; binary32: search).
+//              look-up.
+// LUT = false: no table (16-bit types: packed search; binary32: search).  Which
+// variant runs is decided per call from bits, dtype, activation and n
+// (fewbit_fwd in fewbit_kernels.cu); all give identical codes.
 #pragma once
 
 #include <atomic>
@@ -39,28 +45,14 @@
 
 namespace fewbit {
 
-// threads per CTA: binary32 keeps 32 registers of input in flight per thread, so it runs fewer,
-// fatter threads (register cap 80) than bfloat16 (cap 64)
-#ifndef FEWBIT_LUT_THREADS_BF16
-#define FEWBIT_LUT_THREADS_BF16 512
-#endif
-#ifndef FEWBIT_LUT_CTAS_BF16
-#define FEWBIT_LUT_CTAS_BF16 2
-#endif
+// threads per CTA the kernels are compiled for: binary32 keeps 32 registers of input in flight per
+// thread, so it runs fewer, fatter threads (register cap 80) than the 16-bit types (cap 64); two
+// CTAs of that size are resident per SM.  Variants without a table may be launched with fewer warps.
 #ifndef FEWBIT_LUT_STAGES_BF16
-#define FEWBIT_LUT_STAGES_BF16 1
+#define FEWBIT_LUT_STAGES_BF16 1            // cp.async ring stages of the 16-bit table variant (the table takes 64 KB)
 #endif
-template <typename T, bool LUT = false> struct FwdThreads {
-    static constexpr int value = sizeof(T) == 2 ? (LUT ? FEWBIT_LUT_THREADS_BF16 : 512) : 384;
-};
-#ifndef FEWBIT_CTAS_NOLUT_BF16
-#define FEWBIT_CTAS_NOLUT_BF16 2
-#endif
-constexpr int kFwdCtasPerSm = 2;
-// resident CTAs per SM the kernel is compiled for (register cap = 65536 / threads / this)
-template <typename T, bool LUT> struct FwdCtas {
-    static constexpr int value = sizeof(T) == 2 ? (LUT ? FEWBIT_LUT_CTAS_BF16 : FEWBIT_CTAS_NOLUT_BF16) : kFwdCtasPerSm;
-};
+template <typename T, bool LUT = false> struct FwdThreads { static constexpr int value = sizeof(T) == 2 ? 512 : 384; };
+template <typename T, bool LUT> struct FwdCtas { static constexpr int value = 2; };
 
 template <typename T> constexpr bool kIsHalf = false;
 template <> constexpr bool kIsHalf<__half> = true;
