@@ -189,6 +189,39 @@ def test_config5_sweep_large_sampled(n, dtype):
             del y, p, gi
 
 
+@pytest.mark.parametrize("act", ["gelu", "tanh", "relu"])
+def test_f32_codes_for_every_input_pattern(act, table_mode):
+    """All 2^32 binary32 patterns through fewbit_fwd, 256 M at a time: the packed codes equal
+    #{j : s_j < x} computed by torch.bucketize on the same inputs (NaN -> 0), for every bucketize
+    variant the size-based choice, the forced table and the forced search select."""
+    chunk = 1 << 28
+    base = torch.arange(chunk, device=DEV, dtype=torch.int64)
+    for bits in (2, 3, 4):
+        t = table(act, bits)
+        s_np, _ = t.arrays()
+        bounds = torch.from_numpy(np.ascontiguousarray(s_np)).to(DEV)
+        shifts = torch.arange(0, 32, bits, device=DEV, dtype=torch.int64)[: 32 // bits] if 32 % bits == 0 else None
+        for c in range(16):
+            x = (base + c * chunk).to(torch.int32).view(torch.float32) if c < 8 else \
+                (base + c * chunk - (1 << 32)).to(torch.int32).view(torch.float32)
+            _, pk = fb.fewbit_fwd(t, x)
+            want = torch.bucketize(x, bounds, right=False).to(torch.int64)
+            want = torch.where(torch.isnan(x), torch.zeros_like(want), want)
+            words = pk.view(torch.int32).to(torch.int64) & 0xFFFFFFFF
+            if shifts is not None:                      # 2 and 4 bits: codes do not straddle words
+                got = ((words[:, None] >> shifts[None, :]) & ((1 << bits) - 1)).reshape(-1)
+            else:                                       # 3 bits: 32 codes in 3 words
+                w3 = words.view(-1, 3)
+                bitsream = w3[:, 0] | (w3[:, 1] << 32)  # low 64 bits, then the top word
+                idx = torch.arange(32, device=DEV, dtype=torch.int64) * 3
+                lo = (bitsream[:, None] >> idx[None, :].clamp(max=61)) & 7
+                hi_bits = (w3[:, 1] >> 31) | (w3[:, 2] << 1)      # stream bits 63 ..
+                hi = (hi_bits[:, None] >> (idx[None, :] - 63).clamp(min=0)) & 7
+                got = torch.where(idx[None, :] >= 63, hi, lo).reshape(-1)
+            assert torch.equal(got, want), (act, bits, c)
+            del x, pk, want, words, got
+
+
 def test_more_than_2_to_the_32_elements():
     """Element and word indices beyond 32 bits: 2^32 + 3149 bfloat16 elements (about 28 GB on the
     device), 1 bit (search variant) and 4 bits (table variant, dynamically distributed); sampled
