@@ -481,11 +481,12 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
         }
     }
     constexpr int kFwdThreads = FwdThreads<T, LUT>::value;
-    // Without a table the CTA size is free (a warp's work does not depend on it): 16-bit types run
-    // as 4-warp CTAs, which fill and drain the SMs more evenly on inputs of a few waves.
+    // Without a table the CTA size is free (a warp's work does not depend on it): 4-warp CTAs fill
+    // and drain the SMs more evenly than the 12 or 16 warps the kernel is compiled for (binary32
+    // sigmoid, 51 M elements: 74.7 -> 70.6 us; bfloat16 SiLU, 12.6 M: 15.0 -> 12.9 us).
     size_t warps_per_cta = kFwdThreads / 32;
     if constexpr (!LUT) {
-        if constexpr (sizeof(T) == 2) warps_per_cta = 4;
+        warps_per_cta = 4;
         if (const char *w = fwd_warps_override()) {
             const int v = atoi(w);
             if (v >= 1 && v <= kFwdThreads / 32) warps_per_cta = static_cast<size_t>(v);
@@ -527,10 +528,12 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     const size_t per_cta = warps_per_cta * iters;
     const unsigned grid = static_cast<unsigned>((warp_blocks + per_cta - 1) / per_cta);
     // Programmatic dependent launch lets this grid's CTAs take their places while the previous kernel
-    // of the stream drains (they wait there for it to complete).  Not below one CTA per SM: the
-    // early CTAs land on the SMs the previous kernel left idle, two per SM, and an issue-bound
-    // sub-wave grid then runs on half the SMs (binary32 GELU, 2^20 elements: 8.3 -> 9.2 us).
-    const bool pdl = pdl_enabled() && grid >= static_cast<unsigned>(sms);
+    // of the stream drains (they wait there for it to complete).  Not below one CTA per SM, and for
+    // the issue-bound binary32 activations not below a full wave: the early CTAs pile up on the SMs
+    // the previous kernel left idle, and a sub-wave grid then runs on part of the SMs (binary32
+    // GELU, 2^20 elements: 8.3 -> 9.2 us).
+    const bool issue_bound = sizeof(T) == 4 && act_weight(ACT) == 2;
+    const bool pdl = pdl_enabled() && grid >= static_cast<unsigned>(issue_bound ? slots : static_cast<size_t>(sms));
     return launch_pdl(kernel, grid, static_cast<unsigned>(warps_per_cta * 32), smem * warps_per_cta / (kFwdThreads / 32), st, pdl,
                       prm, static_cast<const T *>(x), static_cast<T *>(y), packed, n, static_cast<int>(iters));
 }
