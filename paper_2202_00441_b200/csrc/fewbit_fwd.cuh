@@ -260,7 +260,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     // global number is congruent to q and hands out the warp-blocks congruent to q (one address
     // alone sustains only ~0.4 G atomics per second; every SM has warps in every group, so the
     // groups finish together).
-    const bool dynamic = LUT && prm.queue != nullptr;
+    const bool dynamic = LUT && prm.queue != nullptr && gridDim.x * warps >= kQueues;   // every counter needs a warp that draws from it
     const size_t full = dynamic ? all_full : (all_full < cta_end ? all_full : cta_end);   // static: this CTA's warp-blocks are [cta_begin, full)
     const uint32_t global_warp = blockIdx.x * static_cast<uint32_t>(warps) + (threadIdx.x >> 5);
     const size_t first_wb = dynamic ? global_warp : warp0;
