@@ -237,7 +237,6 @@ template <int ACT, int BITS, typename T, bool LUT, bool FOLD>
 __global__ void __launch_bounds__(FwdThreads<T, LUT>::value, FwdCtas<T, LUT>::value)
 fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters) {
     pdl_launch_dependents();
-    pdl_wait();
     constexpr bool kIsBf16 = sizeof(T) == 2;
     constexpr int kFwdThreads = FwdThreads<T, LUT>::value;
     constexpr int kCells = kIsBf16 ? (1 << kCellBitsBf16) : (1 << kCellBitsF32);
@@ -285,6 +284,17 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     // With one (shared memory is taken): as soon as a tile of the current warp-block has been
     // consumed, the same registers are reloaded with that tile of the warp's next warp-block, so
     // four loads per lane stay in flight while the warp computes.
+    // The 64 KB table of the 16-bit types is expanded before the wait on the previous kernel of the
+    // stream (it touches shared memory and kernel parameters only), so under programmatic dependent
+    // launch it overlaps that kernel's tail; the 8 KB binary32 table is expanded behind the first
+    // loads instead (its CTAs may be short, and each would pay the serialisation).
+    constexpr bool kExpandFirst = LUT && kIsBf16;
+    if constexpr (kExpandFirst) {
+        FwdSmem &sm = *reinterpret_cast<FwdSmem *>(smem_raw + kCells);
+        if (threadIdx.x < kMaxLevels) sm.thr[threadIdx.x] = prm.tb.s[threadIdx.x];
+        expand_runs<kCells, kFwdThreads>(prm.runs, lut, sm);
+    }
+    pdl_wait();                                                     // nothing above touches global memory
     Raw<T> cur[kTilesPerWarp];
     size_t wb = first_wb;                                           // the warp-block in hand, the one after it,
     size_t nxt = wb < full ? next_after(wb) : full;                 // and (inside the loop) the one after that
@@ -307,7 +317,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
 #pragma unroll
         for (int t = 0; t < kTilesPerWarp; ++t) load_raw(px + t * kTileElems, cur[t]);
     }
-    if constexpr (LUT) {                                            // expanded while the first loads are in flight
+    if constexpr (LUT && !kExpandFirst) {                           // expanded while the first loads are in flight
         FwdSmem &sm = *reinterpret_cast<FwdSmem *>(smem_raw + kCells);
         if (threadIdx.x < kMaxLevels) sm.thr[threadIdx.x] = prm.tb.s[threadIdx.x];
         expand_runs<kCells, kFwdThreads>(prm.runs, lut, sm);
