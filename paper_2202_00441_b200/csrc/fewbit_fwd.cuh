@@ -18,7 +18,9 @@
 //   packed   : 16-bit types -- the same search on TWO elements per
 //              instruction with bf16x2 / f16x2 compares against boundaries
 //              rounded down to the storage type (exact: s < x <=> floor(s) < x
-//              for an x of that type), threshold selection by bitwise masks;
+//              for an x of that type), threshold selection by bitwise masks
+//              (at 4 bits the last pair of boundaries comes from a 64-word
+//              shared-memory table indexed by both 3-bit prefixes);
 //   look-up  : the code is a step function of x, so it is read from a byte
 //              table in shared memory indexed by the top bits of the pattern:
 //                16-bit   : 65 536 entries, one per pattern, the exact code;
@@ -203,7 +205,7 @@ __device__ __forceinline__ uint32_t gt2(uint32_t a, uint32_t b) {          // pe
 __device__ __forceinline__ uint32_t sel2(uint32_t m, uint32_t a, uint32_t b) { return (m & a) | (~m & b); }
 
 template <int BITS, typename T>
-__device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLevels], uint32_t x2) {
+__device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLevels], uint32_t x2, uint32_t pair_table = 0) {
     if constexpr (BITS == 1) {
         return gt2<T>(x2, S[0]) & 0x00010001u;
     } else if constexpr (BITS == 2) {
@@ -221,12 +223,19 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
         const uint32_t m3 = gt2<T>(x2, S[7]);
         const uint32_t m2 = gt2<T>(x2, sel2(m3, S[11], S[3]));
         const uint32_t m1 = gt2<T>(x2, sel2(m2, sel2(m3, S[13], S[5]), sel2(m3, S[9], S[1])));
-        const uint32_t e0 = sel2(m3, S[8], S[0]), e1 = sel2(m3, S[10], S[2]);
-        const uint32_t e2 = sel2(m3, S[12], S[4]), e3 = sel2(m3, S[14], S[6]);
-        const uint32_t m0 = gt2<T>(x2, sel2(m1, sel2(m2, e3, e1), sel2(m2, e2, e0)));
         uint32_t c = m3 & 0x00080008u;
         c |= m2 & 0x00040004u;
         c |= m1 & 0x00020002u;
+        uint32_t last;                                              // the boundaries S[c_lo], S[c_hi] of the last step
+        if (pair_table != 0) {
+            // one shared-memory word indexed by both 3-bit prefixes instead of seven selects
+            asm("ld.shared.u32 %0, [%1];" : "=r"(last) : "r"(pair_table + ((c & 0xeu) << 4) + ((c >> 17) << 2)));
+        } else {
+            const uint32_t e0 = sel2(m3, S[8], S[0]), e1 = sel2(m3, S[10], S[2]);
+            const uint32_t e2 = sel2(m3, S[12], S[4]), e3 = sel2(m3, S[14], S[6]);
+            last = sel2(m1, sel2(m2, e3, e1), sel2(m2, e2, e0));
+        }
+        const uint32_t m0 = gt2<T>(x2, last);
         return c | (m0 & 0x00010001u);
     }
 }
@@ -294,6 +303,16 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         if (threadIdx.x < kMaxLevels) sm.thr[threadIdx.x] = prm.tb.s[threadIdx.x];
         expand_runs<kCells, kFwdThreads>(prm.runs, lut, sm);
     }
+    // 4 bits, packed search: the boundary pair of the last comparison, for every pair of 3-bit
+    // prefixes (low element * 8 + high element), 64 words
+    [[maybe_unused]] uint32_t pair_table = 0;
+    if constexpr (kIsBf16 && !LUT && BITS == 4) {
+        __shared__ uint32_t last_pair[64];
+        if (threadIdx.x < 64)
+            last_pair[threadIdx.x] = (prm.sb2[2 * (threadIdx.x >> 3)] & 0x0000ffffu) | (prm.sb2[2 * (threadIdx.x & 7)] & 0xffff0000u);
+        __syncthreads();
+        pair_table = static_cast<uint32_t>(__cvta_generic_to_shared(last_pair));
+    }
     pdl_wait();                                                     // nothing above touches global memory
     Raw<T> cur[kTilesPerWarp];
     size_t wb = first_wb;                                           // the warp-block in hand, the one after it,
@@ -347,7 +366,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
                     if constexpr (LUT) {
                         pc[e / 2] = lut[cell(cur[t], e)] + (static_cast<uint32_t>(lut[cell(cur[t], e + 1)]) << 16);
                     } else {
-                        pc[e / 2] = bucketize_bf16x2<BITS, T>(prm.sb2, FOLD ? (pair_bits(cur[t], e) & 0x7fff7fffu) : pair_bits(cur[t], e));
+                        pc[e / 2] = bucketize_bf16x2<BITS, T>(prm.sb2, FOLD ? (pair_bits(cur[t], e) & 0x7fff7fffu) : pair_bits(cur[t], e), pair_table);
                     }
                 } else {
                     uint32_t c0, c1;
