@@ -15,6 +15,7 @@ on the data path), time is the max over ranks.
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import statistics
@@ -61,7 +62,7 @@ def measured_peak():
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
 
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -75,12 +76,13 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Summary of the samples; with wall-clock bounds, of those taken between them (the timed region)."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -89,24 +91,41 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
+        rows = []
+        try:
+            rows = open(self.path).read().splitlines()
+            os.unlink(self.path)
+        except Exception:
+            pass
+        out = self._summarise(rows, t_begin, t_end, out, "timed region")
+        if out["samples"] == 0 and t_begin is not None:      # region shorter than the sampling period
+            out = self._summarise(rows, t_begin - 0.25, t_end + 0.25, out, "within 0.25 s of the timed region")
+        return out
+
+    @staticmethod
+    def _summarise(rows, t_begin, t_end, out, window):
         clocks, reasons, mx = [], set(), None
         try:
-            for line in open(self.path):
+            for line in rows:
                 f = [c.strip() for c in line.split(",")]
                 if len(f) < 9:
                     continue
                 try:
+                    if t_begin is not None:
+                        ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                        if not (t_begin <= ts <= t_end):
+                            continue
                     clocks.append(float(f[1])); mx = float(f[2])
                 except ValueError:
                     continue
                 for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                     if v.lower().startswith("active"):
                         reasons.add(name)
-            os.unlink(self.path)
         except Exception:
             pass
         if clocks:
-            out.update(sm_mhz=statistics.median(clocks), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(clocks))
+            out = dict(out, sm_mhz=statistics.median(clocks), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(clocks),
+                       window=window)
         return out
 
 
@@ -272,13 +291,15 @@ def run_ours(args, case: wl.Case, act: str):
         time.sleep(0.25)
     barrier(world)
     launches_before = fb.fewbit_launch_count()
+    t_begin = time.time()
     start.record()
     for s in range(args.steps):
         one_step(ev[s])
     stop.record()
     barrier(world)
+    t_end = time.time()
     launches_in_region = fb.fewbit_launch_count() - launches_before
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     if flush is None:
         total_ms = start.elapsed_time(stop)
     else:                                      # the flush writes are not part of the path: sum the launches
@@ -471,7 +492,7 @@ def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(wl.CONFIGS), default="c3")
