@@ -487,6 +487,35 @@ def test_dynamic_and_static_partition_agree_on_whole_arrays(dtype, monkeypatch):
             assert torch.equal(y0.view(torch.uint8), y1.view(torch.uint8)), (dtype, act, bits)
 
 
+def test_more_streams_than_work_counter_sets_from_several_host_threads(monkeypatch):
+    """24 streams driven by 6 host threads, two table-variant launches each, nothing waited for in
+    between: more launches in flight than there are sets of work counters, so some take the static
+    partition.  Every result equals the search variant's."""
+    n = (1 << 23) + 1024 * 5 + 3
+    t = table("gelu", 4)
+    x = torch.randn(n, device=DEV).mul_(1.7).bfloat16()
+    monkeypatch.setenv("FEWBIT_FWD_TABLE", "never")
+    y_ref, p_ref = fb.fewbit_fwd(t, x)
+    torch.cuda.synchronize()
+    monkeypatch.setenv("FEWBIT_FWD_TABLE", "always")
+    streams = [torch.cuda.Stream() for _ in range(24)]
+    outs = [None] * 48
+
+    def drive(k):
+        torch.cuda.set_device(DEV)
+        for i in range(k, 24, 6):
+            with torch.cuda.stream(streams[i]):
+                outs[2 * i] = fb.fewbit_fwd(t, x)
+                outs[2 * i + 1] = fb.fewbit_fwd(t, x)
+
+    with ThreadPoolExecutor(max_workers=6) as pool:
+        list(pool.map(drive, range(6)))
+    torch.cuda.synchronize()
+    for i, (y, pk) in enumerate(outs):
+        assert torch.equal(pk, p_ref), f"codes differ, launch {i}"
+        assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16)), f"y differs, launch {i}"
+
+
 def test_stream_capture_uses_the_static_partition_and_replays():
     """No work counters are leased while a stream is being captured; the captured launch gives the
     same result as the eager (dynamically distributed) one."""
