@@ -103,6 +103,10 @@ def _load():
         lib.fbo_f64_to_bf16_array.argtypes = [vp, vp, sz]
         lib.fbo_f64_to_f16_array.restype = None
         lib.fbo_f64_to_f16_array.argtypes = [vp, vp, sz]
+        for name in ("fbo_bias_add_f32", "fbo_bias_add_bf16", "fbo_bias_add_f16"):
+            fn = getattr(lib, name)
+            fn.restype = None
+            fn.argtypes = [vp, vp, sz, sz, vp]
         _lib = lib
         return lib
 
@@ -302,6 +306,26 @@ def fwd(name, bits: int, s, x: np.ndarray, fold: bool = False):
     else:
         raise TypeError("x must be float32, float16 or uint16 (bfloat16 bits)")
     return y, packed
+
+
+def bias_add(x: np.ndarray, bias: np.ndarray) -> np.ndarray:
+    """z[r, c] = x[r, c] + bias[c], the exact sum rounded once to the storage type (same dtype
+    convention as ``fwd``: float32, float16, or uint16 holding bfloat16 bits).  ``x`` is
+    (rows, cols) or flat with a length that is a multiple of ``bias.size``."""
+    bias = np.ascontiguousarray(bias)
+    x = np.ascontiguousarray(x)
+    if x.dtype != bias.dtype:
+        raise TypeError("x and bias must have the same dtype")
+    cols = bias.size
+    if cols == 0 or x.size % cols:
+        raise ValueError("x.size must be a multiple of bias.size")
+    z = np.empty_like(x)
+    fn = {np.dtype(np.float32): "fbo_bias_add_f32", np.dtype(np.uint16): "fbo_bias_add_bf16",
+          np.dtype(np.float16): "fbo_bias_add_f16"}.get(x.dtype)
+    if fn is None:
+        raise TypeError("x must be float32, float16 or uint16 (bfloat16 bits)")
+    getattr(_load(), fn)(_ptr(x), _ptr(bias), x.size // cols, cols, _ptr(z))
+    return z
 
 
 def bwd(bits: int, lev, packed: np.ndarray, grad_out: np.ndarray, n: int | None = None):

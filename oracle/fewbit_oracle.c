@@ -31,6 +31,9 @@
  *                             Fig. 3: for an even f' only the positive half-axis
  *                             is quantised, the table lives on [0, B])
  *   fbo_bwd_*                 Listing 1 "backward": grad_in = grad_out * y[code]
+ *   fbo_bias_add_*            an extension in front of Listing 1: the activation's
+ *                             input is x + bias (one bias per column), the exact
+ *                             sum rounded once to the storage type
  *
  * Every function here is pinned by tests/test_oracle_*.py against Table 1,
  * brute force, closed forms and library routines; none is "parity unpinned"
@@ -624,4 +627,35 @@ void fbo_act_deriv_array(int act, const double *x, double *y, size_t n)
 void fbo_f64_to_bf16_array(const double *x, uint16_t *y, size_t n)
 {
     for (size_t e = 0; e < n; ++e) y[e] = fbo_f64_to_bf16(x[e]);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Bias add in front of the activation (an extension: the paper's Listing 1    */
+/* starts at the activation's input).  z[r][c] = x[r][c] + bias[c], the exact  */
+/* sum rounded once to the storage type -- what an unfused framework op that   */
+/* adds the bias and stores the result would hand to the activation.  The sum */
+/* of two binary64 numbers is formed in binary64; it is exact whenever the two */
+/* exponents are less than 29 (binary32) apart, and beyond that the smaller    */
+/* term cannot move the rounding of the larger one, which is itself a value of */
+/* the storage type, so the single rounding below is the IEEE sum.             */
+/* ------------------------------------------------------------------------- */
+void fbo_bias_add_f32(const float *x, const float *bias, size_t rows, size_t cols, float *z)
+{
+    for (size_t r = 0; r < rows; ++r)
+        for (size_t c = 0; c < cols; ++c)
+            z[r * cols + c] = (float)((double)x[r * cols + c] + (double)bias[c]);
+}
+
+void fbo_bias_add_bf16(const uint16_t *x, const uint16_t *bias, size_t rows, size_t cols, uint16_t *z)
+{
+    for (size_t r = 0; r < rows; ++r)
+        for (size_t c = 0; c < cols; ++c)
+            z[r * cols + c] = fbo_f64_to_bf16(fbo_bf16_to_f64(x[r * cols + c]) + fbo_bf16_to_f64(bias[c]));
+}
+
+void fbo_bias_add_f16(const uint16_t *x, const uint16_t *bias, size_t rows, size_t cols, uint16_t *z)
+{
+    for (size_t r = 0; r < rows; ++r)
+        for (size_t c = 0; c < cols; ++c)
+            z[r * cols + c] = fbo_f64_to_f16(fbo_f16_to_f64(x[r * cols + c]) + fbo_f16_to_f64(bias[c]));
 }

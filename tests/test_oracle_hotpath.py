@@ -334,3 +334,92 @@ def test_f16_forward_and_backward_follow_the_same_rules():
     with np.errstate(over="ignore"):
         ref_gi = (g.astype(np.float32) * lev[codes]).astype(np.float64).astype(np.float16)
     np.testing.assert_array_equal(gi.view(np.uint16), ref_gi.view(np.uint16))
+
+
+# --------------------------------------------------------------------------
+# bias add in front of the activation
+# --------------------------------------------------------------------------
+def _rne_to_grid(value: Fraction, grid_vals, grid_bits):
+    """Round an exact rational to the nearest value of a sorted list of representable numbers
+    (ties to the even bit pattern); returns the bit pattern.  Written from the definition."""
+    lo, hi = 0, len(grid_vals) - 1
+    if value <= grid_vals[0]:
+        return grid_bits[0]
+    if value >= grid_vals[-1]:
+        return grid_bits[-1]
+    while hi - lo > 1:
+        mid = (lo + hi) // 2
+        if grid_vals[mid] <= value:
+            lo = mid
+        else:
+            hi = mid
+    dl, dh = value - grid_vals[lo], grid_vals[hi] - value
+    if dl != dh:
+        return grid_bits[lo] if dl < dh else grid_bits[hi]
+    return grid_bits[lo] if grid_bits[lo] % 2 == 0 else grid_bits[hi]
+
+
+def test_bias_add_f32_is_numpy_single_precision_addition():
+    rows, cols = 37, 64
+    x = (RNG.standard_normal((rows, cols)) * 10.0 ** RNG.uniform(-20, 20, (rows, cols))).astype(np.float32)
+    b = (RNG.standard_normal(cols) * 10.0 ** RNG.uniform(-20, 20, cols)).astype(np.float32)
+    x[0, :6] = [0.0, -0.0, np.inf, -np.inf, 1e-45, 3e38]
+    b[:6] = [-0.0, -0.0, -np.inf, 1.0, -1e-45, 3e38]
+    with np.errstate(over="ignore", invalid="ignore"):
+        ref = x + b[None, :]                                  # IEEE binary32 addition, one rounding
+    got = oracle.bias_add(x, b)
+    ok = ~np.isnan(ref)
+    np.testing.assert_array_equal(got.view(np.uint32)[ok], ref.view(np.uint32)[ok])
+    assert np.isnan(got[~ok]).all()
+    # the flat layout is the same thing
+    np.testing.assert_array_equal(oracle.bias_add(x.reshape(-1), b).view(np.uint32)[ok.reshape(-1)],
+                                  ref.reshape(-1).view(np.uint32)[ok.reshape(-1)])
+
+
+def test_bias_add_f16_is_numpy_half_precision_addition_and_the_exact_sum_rounded_once():
+    rows, cols = 64, 1024
+    x = (RNG.standard_normal((rows, cols)) * 10.0 ** RNG.uniform(-6, 4, (rows, cols))).astype(np.float16)
+    b = (RNG.standard_normal(cols) * 10.0 ** RNG.uniform(-6, 4, cols)).astype(np.float16)
+    with np.errstate(over="ignore", invalid="ignore"):
+        ref = x + b[None, :]
+    got = oracle.bias_add(x, b)
+    ok = ~np.isnan(ref)
+    np.testing.assert_array_equal(got.view(np.uint16)[ok], ref.view(np.uint16)[ok])
+    # exact rationals on a subset, ties included: 1 + 2^-11 is half way between two float16 values
+    allh = np.arange(0x7c00, dtype=np.uint16)
+    vals = [Fraction(float(v)) for v in allh.view(np.float16)]
+    grid_vals = [-v for v in vals[:0:-1]] + vals
+    grid_bits = [int(h) | 0x8000 for h in allh[:0:-1]] + [int(h) for h in allh]
+    xs = np.array([1.0, 1.0, 2048.0, -1.0, 6.1e-5, 0.333], dtype=np.float16)
+    bs = np.array([2.0 ** -11, 3 * 2.0 ** -11, 1.0, 2.0 ** -11, 5.96e-8, 0.667], dtype=np.float16)
+    for xv, bv in zip(xs, bs):
+        z = oracle.bias_add(np.array([xv]), np.array([bv]))
+        want = _rne_to_grid(Fraction(float(xv)) + Fraction(float(bv)), grid_vals, grid_bits)
+        assert int(z.view(np.uint16)[0]) == want, (xv, bv)
+
+
+def test_bias_add_bf16_is_the_exact_sum_rounded_once():
+    allh = np.arange(0x7f80, dtype=np.uint16)                # non-negative finite bfloat16 patterns
+    vals = [Fraction(float(v)) for v in bf16_bits_to_f32(allh)]
+    grid_vals = [-v for v in vals[:0:-1]] + vals
+    grid_bits = [int(h) | 0x8000 for h in allh[:0:-1]] + [int(h) for h in allh]
+    n = 600
+    xb = RNG.integers(0x3000, 0x4800, n).astype(np.uint16) | (RNG.integers(0, 2, n).astype(np.uint16) << 15)
+    bb = RNG.integers(0x3000, 0x4800, n).astype(np.uint16) | (RNG.integers(0, 2, n).astype(np.uint16) << 15)
+    # ties: 1 + 2^-8 lies half way between 1 and the next bfloat16; and a pair 30 binades apart
+    xb[:4] = [0x3f80, 0x3f80, 0xbf80, 0x4e80]
+    bb[:4] = [0x3b80, 0x3c40, 0x3b80, 0x3f80]
+    got = oracle.bias_add(xb, bb)                             # one row, n columns
+    for i in range(n):
+        exact = Fraction(float(bf16_bits_to_f32(xb[i:i + 1])[0])) + Fraction(float(bf16_bits_to_f32(bb[i:i + 1])[0]))
+        want = _rne_to_grid(exact, grid_vals, grid_bits)
+        if exact == 0:
+            assert int(got[i]) & 0x7fff == 0
+        else:
+            assert int(got[i]) == want, (hex(xb[i]), hex(bb[i]))
+    # broadcasting over rows: every row gets the same bias
+    x2 = np.tile(xb, (3, 1))
+    np.testing.assert_array_equal(oracle.bias_add(x2, bb), np.tile(got, (3, 1)))
+    # and it equals binary32 addition followed by one rounding to bfloat16 (no double-rounding case exists)
+    f = bf16_bits_to_f32(xb) + bf16_bits_to_f32(bb)
+    np.testing.assert_array_equal(oracle.f64_to_bf16(f.astype(np.float64)), got)
