@@ -368,6 +368,7 @@ def run_ours(args, case: wl.Case, act: str):
         import dataclasses
         f16 = dataclasses.replace(wl.C3, name="c3_shape_f16_2p26", dtype="f16", shape=(1 << 26,), bits=(1, 4))
         also["f16"] = quick_config(fb, f16, dev, reps=5)                   # IEEE binary16 storage
+        also["c2_bias"] = quick_config(fb, wl.C2, dev, bias_cols=wl.C2.shape[-1])   # f(x + bias), the add inside the kernel
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
@@ -437,12 +438,13 @@ def torch_unfused(case: wl.Case, act: str, x, g, reps: int = 5):
             "saved_bytes_per_elem": eb, "note": "stock torch forward + autograd backward, full input kept"}
 
 
-def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False):
+def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False, bias_cols: int = 0):
     """Device-resident timing of another configuration.  L2-cold by rotation: enough independent
     buffer sets that their footprint exceeds 4x the 126 MB L2, a different set for every launch
     (a write-flush would leave the L2 full of dirty lines whose write-back is then charged to a
     kernel that only runs for a few microseconds).  A spin kernel ahead of the first event lets the
-    host finish enqueueing, so the events bracket GPU time, not launch latency."""
+    host finish enqueueing, so the events bracket GPU time, not launch latency.  bias_cols > 0: the
+    forward is fewbit_fwd_bias with a bias of that many columns (f(x + bias), the add fused in)."""
     eb = elem_size(case)
     per_set = case.n * (4 * eb + 0.5)
     sets = max(2, int(512 * 2 ** 20 // per_set) + 1)
@@ -454,6 +456,7 @@ def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False):
     gs = [g0] + [g0.clone() for _ in range(sets - 1)]
     ys = [torch.empty_like(x0) for _ in range(sets)]
     gis = [torch.empty_like(g0) for _ in range(sets)]
+    bias = torch.randn(bias_cols, device=dev).mul_(0.5).to(x0.dtype) if bias_cols else None
     out = {}
     for act in case.acts:
         if folded and act not in ("sigmoid", "tanh"):
@@ -468,7 +471,10 @@ def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False):
                 e[0].record()
                 for j in range(inner):
                     k = (i * inner + j) % sets
-                    fb.fewbit_fwd(t, xs[k], ys[k], ps[k])
+                    if bias is None:
+                        fb.fewbit_fwd(t, xs[k], ys[k], ps[k])
+                    else:
+                        fb.fewbit_fwd_bias(t, xs[k].view(-1, bias_cols), bias, ys[k], ps[k])
                 e[1].record()
                 torch.cuda._sleep(400000)
                 e[2].record()

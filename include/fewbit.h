@@ -207,6 +207,29 @@ FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, vo
                                     uint32_t *packed, size_t n, fewbit_dtype dtype, void *stream);
 
 /*
+ * Forward half with a bias in front of the activation (an extension; Listing 1
+ * starts at the activation's input): for x of shape rows x cols, row-major,
+ *   z[r][c] = x[r][c] + bias[c]     the exact sum, rounded once to `dtype`,
+ *   y = f(z),  code = #{ j : s_j < z }   exactly as fewbit_fwd would on z.
+ * The backward half needs nothing new: grad_in = fewbit_bwd(packed, grad_out)
+ * is the gradient with respect to x, and its column sums are the gradient with
+ * respect to the bias.
+ *
+ * x, y: DEVICE, rows * cols elements; bias: DEVICE, cols elements of `dtype`,
+ * 32-byte aligned like x and y; packed: DEVICE, fewbit_packed_bytes(rows * cols,
+ * bits) bytes, 16-byte aligned.  y may alias x exactly.  cols must be a multiple
+ * of 1024 (one row is then a whole number of the kernel's work units) and the
+ * table must not be a folded one, else FEWBIT_ERR_UNSUPPORTED; rows * cols == 0
+ * is a no-op.  Asynchronous on `stream`, allocates nothing; runs the search
+ * variants of the forward kernel (no code table).
+ * Errors: INVALID_ARG (NULL, bad dtype, rows * cols overflows), UNSUPPORTED,
+ * ALIGNMENT, CUDA.
+ */
+FEWBIT_API fewbit_status fewbit_fwd_bias(const fewbit_table *table, const void *x, const void *bias,
+                                         void *y, uint32_t *packed, size_t rows, size_t cols,
+                                         fewbit_dtype dtype, void *stream);
+
+/*
  * Backward half, one kernel launch on `stream`, asynchronous:
  *     grad_in[e] = round_dtype( (float)grad_out[e] * lev[code[e]] )
  * (Eq. 1 with f' replaced by q of Eq. 2; one binary32 multiply, one rounding).

@@ -64,6 +64,8 @@ def load_library():
     lib.fewbit_packed_bytes.argtypes = [sz, ci]
     lib.fewbit_fwd.restype = ci
     lib.fewbit_fwd.argtypes = [vp, vp, vp, vp, sz, ci, vp]
+    lib.fewbit_fwd_bias.restype = ci
+    lib.fewbit_fwd_bias.argtypes = [vp, vp, vp, vp, vp, sz, sz, ci, vp]
     lib.fewbit_bwd.restype = ci
     lib.fewbit_bwd.argtypes = [vp, vp, vp, vp, sz, ci, vp]
     lib.fewbit_host_workspace_bytes.restype = sz
@@ -234,6 +236,30 @@ def fewbit_fwd(table: Table, x: torch.Tensor, y: Optional[torch.Tensor] = None,
     with torch.cuda.device(x.device):
         _check(lib.fewbit_fwd(table.handle, x.data_ptr(), y.data_ptr(), packed.data_ptr(), n, _DTYPES[x.dtype],
                               _stream_ptr(stream, x.device)), "fewbit_fwd")
+    return y, packed
+
+
+def fewbit_fwd_bias(table: Table, x: torch.Tensor, bias: torch.Tensor, y: Optional[torch.Tensor] = None,
+                    packed: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Forward half of ``f(x + bias)``: ``bias`` has one value per element of the last dimension of
+    ``x`` (a multiple of 1024); returns (y, packed) exactly as ``fewbit_fwd`` would for the tensor
+    ``x + bias`` rounded to the storage type."""
+    lib = load_library()
+    _dev_tensor(x, "x"), _dev_tensor(bias, "bias")
+    n, cols = x.numel(), bias.numel()
+    if bias.dtype != x.dtype or x.dim() == 0 or x.shape[-1] != cols:
+        raise ValueError("bias must have the dtype of x and the length of its last dimension")
+    rows = n // cols if cols else 0
+    if y is None:
+        y = torch.empty_like(x)
+    if packed is None:
+        packed = torch.empty(fewbit_packed_bytes(n, table.bits) // 4, dtype=torch.int32, device=x.device)
+    _dev_tensor(y, "y"), _dev_tensor(packed, "packed")
+    if y.dtype != x.dtype or y.numel() != n or packed.numel() * packed.element_size() < fewbit_packed_bytes(n, table.bits):
+        raise ValueError("y / packed do not match x")
+    with torch.cuda.device(x.device):
+        _check(lib.fewbit_fwd_bias(table.handle, x.data_ptr(), bias.data_ptr(), y.data_ptr(), packed.data_ptr(), rows, cols,
+                                   _DTYPES[x.dtype], _stream_ptr(stream, x.device)), "fewbit_fwd_bias")
     return y, packed
 
 

@@ -93,6 +93,31 @@ __device__ __forceinline__ uint32_t cell(const Raw<__nv_bfloat16> &r, int e) {
 }
 
 // ---------------------------------------------------------------------------
+// optional bias in front of the activation: the lane-chunk becomes x + bias,
+// the exact sum rounded once to the storage type (one IEEE addition in that
+// type: add.rn.f32, add.rn.bf16x2, add.rn.f16x2).
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void add_bias(Raw<float> &r, const float *b) {
+    float v[8];
+    asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(b));
+#pragma unroll
+    for (int e = 0; e < 8; ++e) r.v[e] = __fadd_rn(r.v[e], v[e]);
+}
+__device__ __forceinline__ void add_bias(Raw<__nv_bfloat16> &r, const __nv_bfloat16 *b) {
+    uint32_t v[4];
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "l"(b));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.v[i]) : "r"(r.v[i]), "r"(v[i]));   // one rounding per half
+}
+__device__ __forceinline__ void add_bias(Raw<__half> &r, const __half *b) {
+    uint32_t v[4];
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "l"(b));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) asm("add.rn.f16x2 %0, %1, %2;" : "=r"(r.v[i]) : "r"(r.v[i]), "r"(v[i]));
+}
+
+// ---------------------------------------------------------------------------
 // asynchronous prefetch ring (variants without a code table): every lane copies
 // its own lane-chunks of the next kStages warp-blocks global -> shared with
 // cp.async and reads the same bytes back just before use.  No lane reads what
@@ -189,6 +214,8 @@ struct FwdParams {
     uint32_t sb2[kMaxLevels];        // boundaries rounded down to bfloat16, replicated in both halves
     CodeRuns runs;
     uint32_t *queue;                 // table variants: a leased set of zeroed work counters (dynamic distribution), or NULL (static)
+    const void *bias;                // one value of the storage type per column, added to x before everything else, or NULL
+    uint32_t row_blocks;             // with a bias: warp-blocks per row (the row length is a multiple of kWarpElems)
 };
 
 // ---------------------------------------------------------------------------
@@ -242,7 +269,7 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
 
 // FOLD: the code is the position of |x| (even f', table on [0, B]); the code tables arrive already
 // built that way, the searches strip the sign first.
-template <int ACT, int BITS, typename T, bool LUT, bool FOLD>
+template <int ACT, int BITS, typename T, bool LUT, bool FOLD, bool BIAS = false>
 __global__ void __launch_bounds__(FwdThreads<T, LUT>::value, FwdCtas<T, LUT>::value)
 fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters) {
     pdl_launch_dependents();
@@ -348,10 +375,15 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         const size_t nxt2 = more ? next_after(nxt) : full;
         const T *px_next = x + nxt * kWarpElems + static_cast<size_t>(lane) * kLaneElems;   // read only if `more`
         uint32_t grp[4];
+        // with a bias: this lane's bias values for tile 0 of the warp-block (a row is a whole number of warp-blocks)
+        [[maybe_unused]] const T *bias_row = nullptr;
+        if constexpr (BIAS)
+            bias_row = static_cast<const T *>(prm.bias) + (wb % prm.row_blocks) * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
         if constexpr (kStages > 0) cp_async_wait<(kStages > 0 ? kStages - 1 : 0)>();   // the oldest stage has landed
 #pragma unroll
         for (int t = 0; t < kTilesPerWarp; ++t) {
             if constexpr (kStages > 0) load_raw_shared(ring + stage * kStageBytes + t * (32 * kChunkBytes), cur[t]);
+            if constexpr (BIAS) add_bias(cur[t], bias_row + t * kTileElems);
             float o[8];
             uint32_t g = 0;
             [[maybe_unused]] uint32_t dense = 0;
@@ -490,13 +522,13 @@ const char *fwd_iters_override();        // tuning aid: environment FEWBIT_FWD_I
 bool pdl_enabled();
 const char *fwd_warps_override();        // tuning aid: environment FEWBIT_FWD_WARPS (variant without a table)
 
-template <int ACT, int BITS, typename T, bool LUT, bool FOLD>
+template <int ACT, int BITS, typename T, bool LUT, bool FOLD, bool BIAS = false>
 cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *packed, size_t n, cudaStream_t st) {
     cudaError_t err = cudaSuccess;
     const int sms = device_sm_count(&err);
     if (err != cudaSuccess) return err;
     constexpr size_t smem = fwd_smem_bytes<T, LUT>();
-    auto kernel = fwd_kernel<ACT, BITS, T, LUT, FOLD>;
+    auto kernel = fwd_kernel<ACT, BITS, T, LUT, FOLD, BIAS>;
     if constexpr (smem > 48 * 1024) {           // opt in to the large dynamic shared memory once per device
         static std::atomic<uint64_t> opted_in{0};
         int dev = 0;
@@ -570,7 +602,8 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
 using FwdLaunch = cudaError_t (*)(const FwdParams &, const void *, void *, uint32_t *, size_t, cudaStream_t);
 
 // Launchers of one activation: [bits - 1][dtype: f32, bf16, f16][use look-up table][folded table]
-struct FwdLaunchers { FwdLaunch fn[kMaxBits][3][2][2]; };
+// and, for f(x + bias), the variants without a table and fold: [bits - 1][dtype]
+struct FwdLaunchers { FwdLaunch fn[kMaxBits][3][2][2]; FwdLaunch with_bias[kMaxBits][3]; };
 
 template <int ACT, int BITS, bool FOLD>
 constexpr void fill_fwd_launchers(FwdLaunchers &l) {
@@ -583,6 +616,11 @@ constexpr void fill_fwd_launchers(FwdLaunchers &l) {
     l.fn[BITS - 1][1][1][FOLD] = launch_fwd<ACT, BITS, __nv_bfloat16, kLutBf16, FOLD>;
     l.fn[BITS - 1][2][0][FOLD] = launch_fwd<ACT, BITS, __half, false, FOLD>;
     l.fn[BITS - 1][2][1][FOLD] = launch_fwd<ACT, BITS, __half, kLutBf16, FOLD>;
+    if constexpr (!FOLD) {
+        l.with_bias[BITS - 1][0] = launch_fwd<ACT, BITS, float, false, false, true>;
+        l.with_bias[BITS - 1][1] = launch_fwd<ACT, BITS, __nv_bfloat16, false, false, true>;
+        l.with_bias[BITS - 1][2] = launch_fwd<ACT, BITS, __half, false, false, true>;
+    }
 }
 
 template <int ACT>

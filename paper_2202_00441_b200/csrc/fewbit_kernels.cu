@@ -144,16 +144,16 @@ inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintp
 
 }  // namespace fewbit
 
-extern "C" {
+namespace fewbit {
+namespace {
 
-fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint32_t *packed, size_t n,
-                         fewbit_dtype dtype, void *stream) {
-    using namespace fewbit;
-    if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
-    if (n == 0) return FEWBIT_OK;
-    if (x == nullptr || y == nullptr || packed == nullptr) return FEWBIT_ERR_INVALID_ARG;
-    if (!aligned(x, 32) || !aligned(y, 32) || !aligned(packed, 16)) return FEWBIT_ERR_ALIGNMENT;
+// The forward launch behind fewbit_fwd and fewbit_fwd_bias (bias == nullptr: none; else every row
+// is row_blocks whole warp-blocks long).
+fewbit_status forward(const fewbit_table *table, const void *x, const void *bias, uint32_t row_blocks, void *y,
+                      uint32_t *packed, size_t n, fewbit_dtype dtype, void *stream) {
     FwdParams prm;
+    prm.bias = bias;
+    prm.row_blocks = row_blocks;
     const bool bf16 = dtype != FEWBIT_F32;                              // a 16-bit storage type (same kernel geometry)
     for (int m = 0; m < kMaxLevels; ++m) {
         prm.tb.s[m] = table->s[m];
@@ -186,6 +186,7 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
     // be leased (not during stream capture); the 16-bit types at 3 bits only beat the packed search
     // that way.  binary32 ReLU / leaky ReLU measured faster with short CTAs and a static partition,
     // and below two waves there is nothing to balance.
+    if (bias != nullptr) use_lut = false;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     QueueLease lease;
     const char *queue_mode = getenv("FEWBIT_FWD_QUEUE");               // testing aid: "never" keeps the static partition
@@ -195,7 +196,9 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
         prm.queue = lease.counters;
     }
     if (use_lut && bf16 && table->bits == 3 && prm.queue == nullptr && !forced_table) use_lut = false;
-    const FwdLaunch launch = fwd_launchers(table->act).fn[table->bits - 1][static_cast<int>(dtype)][use_lut][table->folded ? 1 : 0];
+    const FwdLaunchers &all = fwd_launchers(table->act);
+    const FwdLaunch launch = bias != nullptr ? all.with_bias[table->bits - 1][static_cast<int>(dtype)]
+                                             : all.fn[table->bits - 1][static_cast<int>(dtype)][use_lut][table->folded ? 1 : 0];
     if (launch == nullptr) return FEWBIT_ERR_UNSUPPORTED;     // (no lease is held here: the table variants exist whenever runs.count != 0)
     const cudaError_t err = launch(prm, x, y, packed, n, st);
     const cudaError_t rerr = queue_release(lease, st);
@@ -205,6 +208,33 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return FEWBIT_OK;
+}
+
+}  // namespace
+}  // namespace fewbit
+
+extern "C" {
+
+fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint32_t *packed, size_t n,
+                         fewbit_dtype dtype, void *stream) {
+    using namespace fewbit;
+    if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
+    if (n == 0) return FEWBIT_OK;
+    if (x == nullptr || y == nullptr || packed == nullptr) return FEWBIT_ERR_INVALID_ARG;
+    if (!aligned(x, 32) || !aligned(y, 32) || !aligned(packed, 16)) return FEWBIT_ERR_ALIGNMENT;
+    return forward(table, x, nullptr, 0, y, packed, n, dtype, stream);
+}
+
+fewbit_status fewbit_fwd_bias(const fewbit_table *table, const void *x, const void *bias, void *y, uint32_t *packed,
+                              size_t rows, size_t cols, fewbit_dtype dtype, void *stream) {
+    using namespace fewbit;
+    if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return FEWBIT_OK;
+    if (x == nullptr || bias == nullptr || y == nullptr || packed == nullptr) return FEWBIT_ERR_INVALID_ARG;
+    if (cols % kWarpElems != 0 || cols / kWarpElems > 0xffffffffull || table->folded) return FEWBIT_ERR_UNSUPPORTED;
+    if (rows > SIZE_MAX / cols) return FEWBIT_ERR_INVALID_ARG;
+    if (!aligned(x, 32) || !aligned(bias, 32) || !aligned(y, 32) || !aligned(packed, 16)) return FEWBIT_ERR_ALIGNMENT;
+    return forward(table, x, bias, static_cast<uint32_t>(cols / kWarpElems), y, packed, rows * cols, dtype, stream);
 }
 
 fewbit_status fewbit_bwd(const fewbit_table *table, const uint32_t *packed, const void *grad_out, void *grad_in,

@@ -222,6 +222,137 @@ def test_f32_codes_for_every_input_pattern(act, table_mode):
             del x, pk, want, words, got
 
 
+def test_shards_cut_by_shard_range_concatenate_to_the_single_launch_stream():
+    """The multi-GPU path is N independent launches on the ranges `workloads.shard_range` cuts (no
+    exchange step).  Here the shards of a 3- and an 8-way split run one after another on one GPU:
+    their outputs, concatenated, are the single-launch y, packed stream and grad_in, bit for bit."""
+    n = (1 << 22) + 5 * 1024 + 77
+    x = torch.randn(n, device=DEV).mul_(1.5).bfloat16()
+    g = torch.randn(n, device=DEV).bfloat16()
+    for bits in (1, 3, 4):
+        t = table("silu", bits)
+        y, pk = fb.fewbit_fwd(t, x)
+        gi = fb.fewbit_bwd(t, pk, g)
+        for world in (3, 8):
+            ys, pks, gis = [], [], []
+            for rank in range(world):
+                lo, hi = wl.shard_range(n, rank, world)
+                ysh, psh = fb.fewbit_fwd(t, x[lo:hi])
+                gis.append(fb.fewbit_bwd(t, psh, g[lo:hi]))
+                ys.append(ysh)
+                pks.append(psh)
+            torch.cuda.synchronize()
+            assert torch.equal(torch.cat(ys).view(torch.int16), y.view(torch.int16))
+            assert torch.equal(torch.cat(pks), pk), (bits, world)
+            assert torch.equal(torch.cat(gis).view(torch.int16), gi.view(torch.int16))
+
+
+# --------------------------------------------------------------------------
+# bias in front of the activation
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["bf16", "f16", "f32"])
+def test_forward_with_bias_matches_the_oracle(dtype, table_mode):
+    """f(x + bias): the oracle adds the bias (exact sum, one rounding) and runs its forward half on
+    the sum; codes and grad_in bit-exact, y within 2 ulp, for every bucketize variant."""
+    rows, cols = 37, 3072
+    gen = torch.Generator(device=DEV).manual_seed(11)
+    x = (torch.randn(rows, cols, device=DEV, generator=gen) * 1.5).to(TORCH_DT[dtype])
+    b = (torch.randn(cols, device=DEV, generator=gen) * 0.7).to(TORCH_DT[dtype])
+    b[:4] = torch.tensor([0.0, -0.0, 1e-3, -40.0], device=DEV).to(TORCH_DT[dtype])
+    x[0, :8] = torch.tensor([0.0, -0.0, 1.0, -1.0, 65000.0, -1e-7, 3.0, 0.5], device=DEV).to(TORCH_DT[dtype])
+    g = torch.randn(rows, cols, device=DEV, generator=gen).to(TORCH_DT[dtype])
+    z_np = oracle.bias_add(np_bits(x).reshape(rows, cols), np_bits(b)).reshape(-1)
+    for act, bits in (("gelu", 1), ("silu", 2), ("sigmoid", 3), ("gelu", 4), ("tanh", 4)):
+        t = table(act, bits)
+        s_np, lev_np = t.arrays()
+        y, pk = fb.fewbit_fwd_bias(t, x, b)
+        gi = fb.fewbit_bwd(t, pk, g)
+        torch.cuda.synchronize()
+        y_ref, p_ref = oracle.fwd(act, bits, s_np, z_np)
+        gi_ref = oracle.bwd(bits, lev_np, p_ref, np_bits(g).reshape(-1))
+        assert np.array_equal(np_bits(pk).view(np.uint32), p_ref), (dtype, act, bits)
+        assert np.array_equal(np_bits(gi).reshape(-1).view(gi_ref.dtype), gi_ref), (dtype, act, bits)
+        ok = finite_mask(z_np)
+        assert ulp_distance(np_bits(y).reshape(-1)[ok], y_ref[ok]).max() <= 2, (dtype, act, bits)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+def test_bias_sum_over_every_pattern_against_random_patterns(dtype):
+    """Every 16-bit pattern as x (subnormals, infinities, NaNs included), eight rows rolled against
+    a bias of random patterns: the kernel's sum is the oracle's (exact sum, one rounding), seen
+    through the codes (bit-exact) and y (within 2 ulp where the sum is finite)."""
+    cols, rows = 65536, 8
+    rng = np.random.default_rng(77)
+    pat = np.arange(cols, dtype=np.uint16)
+    x_bits = np.stack([np.roll(pat, 8191 * r) for r in range(rows)])
+    b_bits = rng.integers(0, 65536, cols).astype(np.uint16)
+    b_bits[:16] = [0x0000, 0x8000, 0x0001, 0x8001, 0x007f, 0x0080, 0x7f7f, 0xff7f, 0x3f80, 0xbf80, 0x0400, 0x8400, 0x7bff, 0xfbff, 0x3c00, 0xbc00]
+    tdt = TORCH_DT[dtype]
+    x = torch.from_numpy(x_bits.view(np.int16)).to(DEV).view(tdt)
+    b = torch.from_numpy(b_bits.view(np.int16)).to(DEV).view(tdt)
+    as_np = (lambda a: a) if dtype == "bf16" else (lambda a: a.view(np.float16))
+    z_np = oracle.bias_add(as_np(x_bits), as_np(b_bits)).reshape(-1)
+    t = table("silu", 4)
+    s_np, _ = t.arrays()
+    y, pk = fb.fewbit_fwd_bias(t, x, b)
+    torch.cuda.synchronize()
+    y_ref, p_ref = oracle.fwd("silu", 4, s_np, z_np)
+    assert np.array_equal(np_bits(pk).view(np.uint32), p_ref)
+    ok = finite_mask(z_np)
+    assert ulp_distance(np_bits(y).reshape(-1)[ok], y_ref[ok]).max() <= 2
+    # the sum itself, bit for bit: leaky ReLU returns a positive argument unchanged; then the mirror image
+    tl = table("leaky_relu", 1)
+    for flip in (0x0000, 0x8000):
+        xf = torch.from_numpy((x_bits ^ np.uint16(flip)).view(np.int16)).to(DEV).view(tdt)
+        bf = torch.from_numpy((b_bits ^ np.uint16(flip)).view(np.int16)).to(DEV).view(tdt)
+        zf = oracle.bias_add(as_np(x_bits ^ np.uint16(flip)), as_np(b_bits ^ np.uint16(flip))).reshape(-1)
+        yl, _ = fb.fewbit_fwd_bias(tl, xf, bf)
+        torch.cuda.synchronize()
+        zv = bf16_bits_to_f32(zf) if dtype == "bf16" else zf.astype(np.float32)
+        pos = np.isfinite(zv) & (zv > 0)
+        assert pos.sum() > 100000
+        assert np.array_equal(np_bits(yl).reshape(-1).view(np.uint16)[pos], zf.view(np.uint16)[pos])
+
+
+def test_autograd_layer_with_bias_gives_the_column_sums():
+    rows, cols = 48, 2048
+    x = torch.randn(rows, cols, device=DEV, dtype=torch.bfloat16, requires_grad=True)
+    bias = (torch.randn(cols, device=DEV) * 0.5).bfloat16().requires_grad_(True)
+    layer = fb.FewBitActivation("gelu", bits=3)
+    y = layer(x, bias)
+    g = torch.randn_like(y)
+    y.backward(g)
+    t = layer.table
+    z = (x.detach().float() + bias.detach().float()[None, :]).bfloat16()
+    y_ref, pk = fb.fewbit_fwd(t, z)
+    gi_ref = fb.fewbit_bwd(t, pk, g)
+    assert torch.equal(y.detach().view(torch.int16), y_ref.view(torch.int16))
+    assert torch.equal(x.grad.view(torch.int16), gi_ref.view(torch.int16))
+    assert torch.equal(bias.grad, gi_ref.float().sum(0).bfloat16())
+
+
+def test_forward_with_bias_on_a_large_tensor_in_place_and_its_argument_checks():
+    rows, cols = 8192, 4096                               # 2^25 elements: the dynamically distributed table variant at 4 bits
+    t = table("gelu", 4)
+    x = torch.randn(rows, cols, device=DEV).bfloat16()
+    b = torch.randn(cols, device=DEV).bfloat16()
+    y, pk = fb.fewbit_fwd_bias(t, x, b)
+    z = (x.float() + b.float()[None, :]).bfloat16()       # binary32 sum, one rounding: the same value
+    y2, pk2 = fb.fewbit_fwd(t, z)
+    torch.cuda.synchronize()
+    assert torch.equal(pk, pk2) and torch.equal(y.view(torch.int16), y2.view(torch.int16))
+    xi = x.clone()
+    fb.fewbit_fwd_bias(t, xi, b, y=xi)                    # y aliases x
+    torch.cuda.synchronize()
+    assert torch.equal(xi.view(torch.int16), y.view(torch.int16))
+    compare_sampled("gelu", 4, z.reshape(-1), z.reshape(-1), y.reshape(-1), pk, fb.fewbit_bwd(t, pk, z.reshape(-1)), "bias, large")
+    with pytest.raises(fb.FewbitError) as e:              # a row must be a whole number of 1024-element blocks
+        fb.fewbit_fwd_bias(t, x[:, :1000].contiguous(), b[:1000].contiguous())
+    assert e.value.status == 2
+    with pytest.raises(ValueError):
+        fb.fewbit_fwd_bias(t, x, b[:1024].contiguous())
+
+
 def test_more_than_2_to_the_32_elements():
     """Element and word indices beyond 32 bits: 2^32 + 3149 bfloat16 elements (about 28 GB on the
     device), 1 bit (search variant) and 4 bits (table variant, dynamically distributed); sampled
