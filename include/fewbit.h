@@ -220,8 +220,8 @@ FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, vo
  * bits) bytes, 16-byte aligned.  y may alias x exactly.  cols must be a multiple
  * of 1024 (one row is then a whole number of the kernel's work units) and the
  * table must not be a folded one, else FEWBIT_ERR_UNSUPPORTED; rows * cols == 0
- * is a no-op.  Asynchronous on `stream`, allocates nothing; runs the search
- * variants of the forward kernel (no code table).
+ * is a no-op.  Asynchronous on `stream`, allocates nothing; same kernel
+ * variants and launch rules as fewbit_fwd.
  * Errors: INVALID_ARG (NULL, bad dtype, rows * cols overflows), UNSUPPORTED,
  * ALIGNMENT, CUDA.
  */

@@ -602,8 +602,8 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
 using FwdLaunch = cudaError_t (*)(const FwdParams &, const void *, void *, uint32_t *, size_t, cudaStream_t);
 
 // Launchers of one activation: [bits - 1][dtype: f32, bf16, f16][use look-up table][folded table]
-// and, for f(x + bias), the variants without a table and fold: [bits - 1][dtype]
-struct FwdLaunchers { FwdLaunch fn[kMaxBits][3][2][2]; FwdLaunch with_bias[kMaxBits][3]; };
+// and, for f(x + bias) (no folded tables): [bits - 1][dtype][use look-up table]
+struct FwdLaunchers { FwdLaunch fn[kMaxBits][3][2][2]; FwdLaunch with_bias[kMaxBits][3][2]; };
 
 template <int ACT, int BITS, bool FOLD>
 constexpr void fill_fwd_launchers(FwdLaunchers &l) {
@@ -617,9 +617,12 @@ constexpr void fill_fwd_launchers(FwdLaunchers &l) {
     l.fn[BITS - 1][2][0][FOLD] = launch_fwd<ACT, BITS, __half, false, FOLD>;
     l.fn[BITS - 1][2][1][FOLD] = launch_fwd<ACT, BITS, __half, kLutBf16, FOLD>;
     if constexpr (!FOLD) {
-        l.with_bias[BITS - 1][0] = launch_fwd<ACT, BITS, float, false, false, true>;
-        l.with_bias[BITS - 1][1] = launch_fwd<ACT, BITS, __nv_bfloat16, false, false, true>;
-        l.with_bias[BITS - 1][2] = launch_fwd<ACT, BITS, __half, false, false, true>;
+        l.with_bias[BITS - 1][0][0] = launch_fwd<ACT, BITS, float, false, false, true>;
+        l.with_bias[BITS - 1][0][1] = launch_fwd<ACT, BITS, float, kLutF32, false, true>;
+        l.with_bias[BITS - 1][1][0] = launch_fwd<ACT, BITS, __nv_bfloat16, false, false, true>;
+        l.with_bias[BITS - 1][1][1] = launch_fwd<ACT, BITS, __nv_bfloat16, kLutBf16, false, true>;
+        l.with_bias[BITS - 1][2][0] = launch_fwd<ACT, BITS, __half, false, false, true>;
+        l.with_bias[BITS - 1][2][1] = launch_fwd<ACT, BITS, __half, kLutBf16, false, true>;
     }
 }
 
