@@ -72,6 +72,7 @@ cudaError_t queue_acquire(cudaStream_t stream, QueueLease *lease) {
         const cudaError_t q = cudaEventQuery(st.slot[i].done);
         if (q == cudaSuccess) pick = i;
         else if (q != cudaErrorNotReady) return q;
+        else (void)cudaGetLastError();       // "not ready" is an answer, not an error: do not leave it behind for a later cudaGetLastError
     }
     if (pick < 0) return cudaSuccess;
     Slot &s = st.slot[pick];
