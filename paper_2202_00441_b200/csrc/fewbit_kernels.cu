@@ -186,6 +186,12 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
     // be leased (not during stream capture); the 16-bit types at 3 bits only beat the packed search
     // that way.  binary32 ReLU / leaky ReLU measured faster with short CTAs and a static partition,
     // and below two waves there is nothing to balance.
+    const FwdLaunchers &all = fwd_launchers(table->act);
+    auto launcher = [&](bool lut) {
+        return bias != nullptr ? all.with_bias[table->bits - 1][static_cast<int>(dtype)][lut]
+                               : all.fn[table->bits - 1][static_cast<int>(dtype)][lut][table->folded ? 1 : 0];
+    };
+    if (launcher(use_lut) == nullptr || launcher(false) == nullptr) return FEWBIT_ERR_UNSUPPORTED;   // before any lease is taken
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     QueueLease lease;
     const char *queue_mode = getenv("FEWBIT_FWD_QUEUE");               // testing aid: "never" keeps the static partition
@@ -195,11 +201,7 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
         prm.queue = lease.counters;
     }
     if (use_lut && bf16 && table->bits == 3 && prm.queue == nullptr && !forced_table) use_lut = false;
-    const FwdLaunchers &all = fwd_launchers(table->act);
-    const FwdLaunch launch = bias != nullptr ? all.with_bias[table->bits - 1][static_cast<int>(dtype)][use_lut]
-                                             : all.fn[table->bits - 1][static_cast<int>(dtype)][use_lut][table->folded ? 1 : 0];
-    if (launch == nullptr) return FEWBIT_ERR_UNSUPPORTED;     // (no lease is held here: the table variants exist whenever runs.count != 0)
-    const cudaError_t err = launch(prm, x, y, packed, n, st);
+    const cudaError_t err = launcher(use_lut)(prm, x, y, packed, n, st);
     const cudaError_t rerr = queue_release(lease, st);
     if (err != cudaSuccess || rerr != cudaSuccess) {
         t_last_cuda_error = static_cast<int>(err != cudaSuccess ? err : rerr);
