@@ -216,6 +216,7 @@ struct FwdParams {
     uint32_t *queue;                 // table variants: a leased set of zeroed work counters (dynamic distribution), or NULL (static)
     const void *bias;                // one value of the storage type per column, added to x before everything else, or NULL
     uint32_t row_blocks;             // with a bias: warp-blocks per row (the row length is a multiple of kWarpElems)
+    uint32_t long_iters;             // warp-blocks per warp of the long CTAs of a static partition
 };
 
 // ---------------------------------------------------------------------------
@@ -271,7 +272,7 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
 // built that way, the searches strip the sign first.
 template <int ACT, int BITS, typename T, bool LUT, bool FOLD, bool BIAS = false>
 __global__ void __launch_bounds__(FwdThreads<T, LUT>::value, FwdCtas<T, LUT>::value)
-fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters) {
+fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters, unsigned long_ctas) {
     pdl_launch_dependents();
     constexpr bool kIsBf16 = sizeof(T) == 2;
     constexpr int kFwdThreads = FwdThreads<T, LUT>::value;
@@ -282,7 +283,13 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
 
     const int lane = threadIdx.x & 31;
     const size_t warps = blockDim.x >> 5;                                        // stride between a warp's warp-blocks (<= kFwdThreads / 32)
-    const size_t cta_begin = static_cast<size_t>(blockIdx.x) * warps * iters;
+    // Static partition: the first long_ctas CTAs own warps * iters warp-blocks each, the rest of the
+    // grid warps * 1 (short CTAs at the end of the launch order fill the tail that the long ones
+    // leave when they finish at different times).
+    if (blockIdx.x >= long_ctas) iters = 1;
+    const size_t cta_begin = blockIdx.x < long_ctas
+        ? static_cast<size_t>(blockIdx.x) * warps * iters
+        : static_cast<size_t>(long_ctas) * warps * prm.long_iters + static_cast<size_t>(blockIdx.x - long_ctas) * warps;
     const size_t warp0 = cta_begin + (threadIdx.x >> 5);
     const size_t all_full = n / kWarpElems;
     const size_t cta_end = cta_begin + warps * iters;
@@ -586,8 +593,23 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
         iters = iters < 1 ? 1 : (iters > 4 ? 4 : iters);
     }
     if (const char *dbg = fwd_iters_override()) iters = static_cast<size_t>(atoi(dbg));
+    // When the CTAs take several warp-blocks per warp, the last wave's worth of warp-blocks goes to
+    // short CTAs (one warp-block per warp) at the end of the launch order: they fill the tail that
+    // the long CTAs leave when they finish at different times (2^26 elements: 50.2 -> 48.1 us,
+    // 2^28: 171 -> 169 us).  Without a table only (a table variant is one wave).
     const size_t per_cta = warps_per_cta * iters;
-    const unsigned grid = static_cast<unsigned>((warp_blocks + per_cta - 1) / per_cta);
+    size_t short_blocks = 0;
+    if (!LUT && iters > 1) {
+        short_blocks = warps_per_cta * slots;
+        if (short_blocks > warp_blocks) short_blocks = warp_blocks;
+    }
+    const size_t long_ctas = (warp_blocks - short_blocks) / per_cta;
+    const size_t rest = warp_blocks - long_ctas * per_cta;               // done by short CTAs (or, if none are wanted, one more long one)
+    const size_t short_ctas = short_blocks ? (rest + warps_per_cta - 1) / warps_per_cta : (rest + per_cta - 1) / per_cta;
+    const unsigned grid = static_cast<unsigned>(long_ctas + short_ctas);
+    FwdParams p2 = prm;
+    p2.long_iters = static_cast<uint32_t>(iters);
+    const unsigned n_long = short_blocks ? static_cast<unsigned>(long_ctas) : grid;
     // Programmatic dependent launch lets this grid's CTAs take their places while the previous kernel
     // of the stream drains (they wait there for it to complete).  Not below one CTA per SM, and for
     // the issue-bound binary32 activations not below a full wave: the early CTAs pile up on the SMs
@@ -596,7 +618,7 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     const bool issue_bound = sizeof(T) == 4 && act_weight(ACT) == 2;
     const bool pdl = pdl_enabled() && grid >= static_cast<unsigned>(issue_bound ? slots : static_cast<size_t>(sms));
     return launch_pdl(kernel, grid, static_cast<unsigned>(warps_per_cta * 32), smem * warps_per_cta / (kFwdThreads / 32), st, pdl,
-                      prm, static_cast<const T *>(x), static_cast<T *>(y), packed, n, static_cast<int>(iters));
+                      p2, static_cast<const T *>(x), static_cast<T *>(y), packed, n, static_cast<int>(iters), n_long);
 }
 
 using FwdLaunch = cudaError_t (*)(const FwdParams &, const void *, void *, uint32_t *, size_t, cudaStream_t);
