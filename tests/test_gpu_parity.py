@@ -351,6 +351,19 @@ def test_forward_with_bias_on_a_large_tensor_in_place_and_its_argument_checks():
     assert e.value.status == 2
     with pytest.raises(ValueError):
         fb.fewbit_fwd_bias(t, x, b[:1024].contiguous())
+    with pytest.raises(fb.FewbitError) as e:              # no folded tables with a bias
+        fb.fewbit_fwd_bias(fb.fewbit_table_create_folded("tanh", 2), x, b)
+    assert e.value.status == 2
+    # binary32 at a size where its table variant is distributed dynamically (3 and 4 bits)
+    xf = torch.randn(4096, 4096, device=DEV)
+    bf = torch.randn(4096, device=DEV)
+    zf = xf + bf[None, :]                                 # one IEEE binary32 addition per element
+    for act, bits in (("sigmoid", 3), ("silu", 4)):
+        tf = table(act, bits)
+        y1, p1 = fb.fewbit_fwd_bias(tf, xf, bf)
+        y2, p2 = fb.fewbit_fwd(tf, zf)
+        torch.cuda.synchronize()
+        assert torch.equal(p1, p2) and torch.equal(y1.view(torch.int32), y2.view(torch.int32)), (act, bits)
 
 
 def test_more_than_2_to_the_32_elements():
