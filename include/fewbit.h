@@ -218,9 +218,9 @@ FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, vo
  * x, y: DEVICE, rows * cols elements; bias: DEVICE, cols elements of `dtype`,
  * 32-byte aligned like x and y; packed: DEVICE, fewbit_packed_bytes(rows * cols,
  * bits) bytes, 16-byte aligned.  y may alias x exactly.  cols must be a multiple
- * of 1024 (one row is then a whole number of the kernel's work units) and the
- * table must not be a folded one, else FEWBIT_ERR_UNSUPPORTED; rows * cols == 0
- * is a no-op.  Asynchronous on `stream`, allocates nothing; same kernel
+ * of 8 below 2^32 (a lane's 8 consecutive elements then never straddle a row
+ * end) and the table must not be a folded one, else FEWBIT_ERR_UNSUPPORTED;
+ * rows * cols == 0 is a no-op.  Asynchronous on `stream`, allocates nothing; same kernel
  * variants and launch rules as fewbit_fwd.
  * Errors: INVALID_ARG (NULL, bad dtype, rows * cols overflows), UNSUPPORTED,
  * ALIGNMENT, CUDA.

@@ -76,7 +76,7 @@ class FewBitActivation(nn.Module):
 
     def forward(self, x: torch.Tensor, bias: torch.Tensor | None = None) -> torch.Tensor:
         """``bias`` (optional): one value per element of the last dimension of ``x`` (a multiple of
-        1024), added to ``x`` inside the kernel."""
+        8), added to ``x`` inside the kernel."""
         if bias is not None:
             return _FewBitBiasFunction.apply(x, bias, self.table)
         return _FewBitFunction.apply(x, self.table)

@@ -242,7 +242,7 @@ def fewbit_fwd(table: Table, x: torch.Tensor, y: Optional[torch.Tensor] = None,
 def fewbit_fwd_bias(table: Table, x: torch.Tensor, bias: torch.Tensor, y: Optional[torch.Tensor] = None,
                     packed: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
     """Forward half of ``f(x + bias)``: ``bias`` has one value per element of the last dimension of
-    ``x`` (a multiple of 1024); returns (y, packed) exactly as ``fewbit_fwd`` would for the tensor
+    ``x`` (a multiple of 8); returns (y, packed) exactly as ``fewbit_fwd`` would for the tensor
     ``x + bias`` rounded to the storage type."""
     lib = load_library()
     _dev_tensor(x, "x"), _dev_tensor(bias, "bias")

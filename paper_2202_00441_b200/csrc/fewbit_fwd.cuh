@@ -97,6 +97,11 @@ __device__ __forceinline__ uint32_t cell(const Raw<__nv_bfloat16> &r, int e) {
 // the exact sum rounded once to the storage type (one IEEE addition in that
 // type: add.rn.f32, add.rn.bf16x2, add.rn.f16x2).
 // ---------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float round_to(float v) {     // v rounded to T (nearest even), widened back
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) return __bfloat162float(__float2bfloat16_rn(v));
+    else if constexpr (std::is_same<T, __half>::value) return __half2float(__float2half_rn(v));
+    else return v;
+}
 __device__ __forceinline__ void add_bias(Raw<float> &r, const float *b) {
     float v[8];
     asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
@@ -215,7 +220,8 @@ struct FwdParams {
     CodeRuns runs;
     uint32_t *queue;                 // table variants: a leased set of zeroed work counters (dynamic distribution), or NULL (static)
     const void *bias;                // one value of the storage type per column, added to x before everything else, or NULL
-    uint32_t row_blocks;             // with a bias: warp-blocks per row (the row length is a multiple of kWarpElems)
+    uint32_t cols;                   // with a bias: the row length, a multiple of kLaneElems (a lane-chunk never straddles a row end)
+    uint64_t chunks_magic;           // floor(2^64 / (cols / kLaneElems)) + 1: exact division of 32-bit chunk numbers by a multiply-high
     uint32_t long_iters;             // warp-blocks per warp of the long CTAs of a static partition
 };
 
@@ -383,14 +389,30 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         const T *px_next = x + nxt * kWarpElems + static_cast<size_t>(lane) * kLaneElems;   // read only if `more`
         uint32_t grp[4];
         // with a bias: this lane's bias values for tile 0 of the warp-block (a row is a whole number of warp-blocks)
-        [[maybe_unused]] const T *bias_row = nullptr;
-        if constexpr (BIAS)
-            bias_row = static_cast<const T *>(prm.bias) + (wb % prm.row_blocks) * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
+        // with a bias: the column of this lane's chunk in tile 0 of the warp-block (one 64-bit remainder
+        // per warp-block; the tiles that follow add 256 and wrap around the row end)
+        [[maybe_unused]] uint64_t col0 = 0;
+        [[maybe_unused]] bool one_row = false;                      // the whole warp-block lies in one row (warp-uniform)
+        if constexpr (BIAS) {
+            const uint64_t chunk = wb * (kWarpElems / kLaneElems);          // number of the warp-block's first lane-chunk
+            const uint32_t row_chunks = prm.cols / kLaneElems;
+            const uint64_t rem = chunk < (1ull << 32) ? chunk - __umul64hi(chunk, prm.chunks_magic) * row_chunks : chunk % row_chunks;
+            one_row = (rem + kWarpElems / kLaneElems) * kLaneElems <= prm.cols;
+            col0 = (rem + lane) * kLaneElems;
+        }
         if constexpr (kStages > 0) cp_async_wait<(kStages > 0 ? kStages - 1 : 0)>();   // the oldest stage has landed
 #pragma unroll
         for (int t = 0; t < kTilesPerWarp; ++t) {
             if constexpr (kStages > 0) load_raw_shared(ring + stage * kStageBytes + t * (32 * kChunkBytes), cur[t]);
-            if constexpr (BIAS) add_bias(cur[t], bias_row + t * kTileElems);
+            if constexpr (BIAS) {
+                if (one_row) {
+                    add_bias(cur[t], static_cast<const T *>(prm.bias) + col0 + t * kTileElems);
+                } else {
+                    uint64_t col = col0 + static_cast<uint64_t>(t) * kTileElems;
+                    if (col >= prm.cols) col = prm.cols >= kWarpElems ? col - prm.cols : col % prm.cols;
+                    add_bias(cur[t], static_cast<const T *>(prm.bias) + col);
+                }
+            }
             float o[8];
             uint32_t g = 0;
             [[maybe_unused]] uint32_t dense = 0;
@@ -476,7 +498,9 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
             if (base + e < n) {
-                const float xv = load1(x + base + e);
+                float xv = load1(x + base + e);
+                if constexpr (BIAS)                                  // the sum rounded once to the storage type
+                    xv = round_to<T>(__fadd_rn(xv, load1(static_cast<const T *>(prm.bias) + (base + e) % prm.cols)));
                 store1(y + base + e, activation<ACT, T>(xv));
                 const uint32_t c = bucketize<BITS>(prm.tb, FOLD ? fabsf(xv) : xv);
                 const int pos = e * BITS;

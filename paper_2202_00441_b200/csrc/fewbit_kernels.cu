@@ -147,13 +147,14 @@ inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintp
 namespace fewbit {
 namespace {
 
-// The forward launch behind fewbit_fwd and fewbit_fwd_bias (bias == nullptr: none; else every row
-// is row_blocks whole warp-blocks long).
-fewbit_status forward(const fewbit_table *table, const void *x, const void *bias, uint32_t row_blocks, void *y,
+// The forward launch behind fewbit_fwd and fewbit_fwd_bias (bias == nullptr: none; else rows of
+// `cols` elements, a multiple of the lane-chunk).
+fewbit_status forward(const fewbit_table *table, const void *x, const void *bias, uint32_t cols, void *y,
                       uint32_t *packed, size_t n, fewbit_dtype dtype, void *stream) {
     FwdParams prm;
     prm.bias = bias;
-    prm.row_blocks = row_blocks;
+    prm.cols = cols;
+    prm.chunks_magic = cols > static_cast<uint32_t>(kLaneElems) ? ~0ull / (cols / kLaneElems) + 1 : 0;   // one chunk per row: remainder 0
     const bool bf16 = dtype != FEWBIT_F32;                              // a 16-bit storage type (same kernel geometry)
     for (int m = 0; m < kMaxLevels; ++m) {
         prm.tb.s[m] = table->s[m];
@@ -232,10 +233,10 @@ fewbit_status fewbit_fwd_bias(const fewbit_table *table, const void *x, const vo
     if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return FEWBIT_OK;
     if (x == nullptr || bias == nullptr || y == nullptr || packed == nullptr) return FEWBIT_ERR_INVALID_ARG;
-    if (cols % kWarpElems != 0 || cols / kWarpElems > 0xffffffffull || table->folded) return FEWBIT_ERR_UNSUPPORTED;
+    if (cols % kLaneElems != 0 || cols > 0xffffffffull || table->folded) return FEWBIT_ERR_UNSUPPORTED;
     if (rows > SIZE_MAX / cols) return FEWBIT_ERR_INVALID_ARG;
     if (!aligned(x, 32) || !aligned(bias, 32) || !aligned(y, 32) || !aligned(packed, 16)) return FEWBIT_ERR_ALIGNMENT;
-    return forward(table, x, bias, static_cast<uint32_t>(cols / kWarpElems), y, packed, rows * cols, dtype, stream);
+    return forward(table, x, bias, static_cast<uint32_t>(cols), y, packed, rows * cols, dtype, stream);
 }
 
 fewbit_status fewbit_bwd(const fewbit_table *table, const uint32_t *packed, const void *grad_out, void *grad_in,

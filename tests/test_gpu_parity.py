@@ -276,6 +276,29 @@ def test_forward_with_bias_matches_the_oracle(dtype, table_mode):
         assert ulp_distance(np_bits(y).reshape(-1)[ok], y_ref[ok]).max() <= 2, (dtype, act, bits)
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("rows,cols", [(3, 8), (129, 40), (77, 1000), (5, 11008), (1, 1048), (1031, 1016)])
+def test_forward_with_bias_on_row_lengths_that_are_not_whole_warp_blocks(dtype, rows, cols, table_mode):
+    """Row lengths that are multiples of 8 only: warp-blocks straddle row ends, the last one is
+    ragged and takes the scalar path; codes and grad_in bit-exact, y within 2 ulp."""
+    gen = torch.Generator(device=DEV).manual_seed(rows * 131 + cols)
+    x = (torch.randn(rows, cols, device=DEV, generator=gen) * 1.5).to(TORCH_DT[dtype])
+    b = torch.randn(cols, device=DEV, generator=gen).to(TORCH_DT[dtype])
+    g = torch.randn(rows, cols, device=DEV, generator=gen).to(TORCH_DT[dtype])
+    z_np = oracle.bias_add(np_bits(x).reshape(rows, cols), np_bits(b)).reshape(-1)
+    for act, bits in (("silu", 1), ("gelu", 3), ("tanh", 4)):
+        t = table(act, bits)
+        s_np, lev_np = t.arrays()
+        y, pk = fb.fewbit_fwd_bias(t, x, b)
+        gi = fb.fewbit_bwd(t, pk, g)
+        torch.cuda.synchronize()
+        y_ref, p_ref = oracle.fwd(act, bits, s_np, z_np)
+        gi_ref = oracle.bwd(bits, lev_np, p_ref, np_bits(g).reshape(-1))
+        assert np.array_equal(np_bits(pk).view(np.uint32), p_ref), (dtype, rows, cols, act, bits)
+        assert np.array_equal(np_bits(gi).reshape(-1).view(gi_ref.dtype), gi_ref)
+        assert ulp_distance(np_bits(y).reshape(-1), y_ref).max() <= 2
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f16"])
 def test_bias_sum_over_every_pattern_against_random_patterns(dtype):
     """Every 16-bit pattern as x (subnormals, infinities, NaNs included), eight rows rolled against
@@ -315,7 +338,7 @@ def test_bias_sum_over_every_pattern_against_random_patterns(dtype):
 
 
 def test_autograd_layer_with_bias_gives_the_column_sums():
-    rows, cols = 48, 2048
+    rows, cols = 48, 2056
     x = torch.randn(rows, cols, device=DEV, dtype=torch.bfloat16, requires_grad=True)
     bias = (torch.randn(cols, device=DEV) * 0.5).bfloat16().requires_grad_(True)
     layer = fb.FewBitActivation("gelu", bits=3)
@@ -346,8 +369,8 @@ def test_forward_with_bias_on_a_large_tensor_in_place_and_its_argument_checks():
     torch.cuda.synchronize()
     assert torch.equal(xi.view(torch.int16), y.view(torch.int16))
     compare_sampled("gelu", 4, z.reshape(-1), z.reshape(-1), y.reshape(-1), pk, fb.fewbit_bwd(t, pk, z.reshape(-1)), "bias, large")
-    with pytest.raises(fb.FewbitError) as e:              # a row must be a whole number of 1024-element blocks
-        fb.fewbit_fwd_bias(t, x[:, :1000].contiguous(), b[:1000].contiguous())
+    with pytest.raises(fb.FewbitError) as e:              # a row must be a whole number of 8-element lane-chunks
+        fb.fewbit_fwd_bias(t, x[:, :1004].contiguous(), b[:1004].contiguous())
     assert e.value.status == 2
     with pytest.raises(ValueError):
         fb.fewbit_fwd_bias(t, x, b[:1024].contiguous())
