@@ -543,10 +543,10 @@ constexpr size_t fwd_smem_bytes() {
 int device_sm_count(cudaError_t *err);   // of the current device, cached
 
 // How much arithmetic an activation costs in binary32: 0 = a few instructions (ReLU, leaky ReLU),
-// 1 = one exponential or tanh, 2 = enough to make the forward kernel issue-bound (GELU, SiLU, softplus).
+// 1 = one exponential or tanh, 2 = enough to make the forward kernel issue-bound (GELU, SiLU).
 constexpr int act_weight(int act) {
     return (act == FEWBIT_RELU || act == FEWBIT_LEAKY_RELU) ? 0
-         : (act == FEWBIT_GELU || act == FEWBIT_SILU || act == FEWBIT_SOFTPLUS) ? 2 : 1;
+         : (act == FEWBIT_GELU || act == FEWBIT_SILU) ? 2 : 1;
 }
 constexpr size_t kLutMinIters = 8;      // below this many warp-blocks per warp the table does not pay for its expansion
 const char *fwd_iters_override();        // tuning aid: environment FEWBIT_FWD_ITERS

@@ -307,8 +307,24 @@ __device__ __forceinline__ float2 act_f32(float2 x) {
         const float2 m = expm1_nonpos_f32(make_float2(fminf(x.x, 0.0f), fminf(x.y, 0.0f)));
         return make_float2(x.x > 0.0f ? x.x : m.x, x.y > 0.0f ? x.y : m.y);
     } else if constexpr (ACT == FEWBIT_SOFTPLUS) {
+        // max(x,0) + log(1 + E),  E = e^{-|x|} in (0, 1]:  log(1 + E) = 2 atanh(s),  s = E / (2 + E) <= 1/3.
+        // The sum 2 + E is kept as d + dl (exact), the quotient gets one Newton step with the
+        // residual E - (d + dl) s0, and atanh(s) = s + s^3 P(s^2) with P of degree 4 (1e-10).
         const float2 e = mul2(exp_scaled_f32(make_float2(-fabsf(x.x), -fabsf(x.y))), splat(kScaleDown));
-        return add2(relu2(x), make_float2(log1pf(e.x), log1pf(e.y)));
+        const float2 d = add2(e, splat(2.0f));
+        const float2 nd = fma2(e, splat(-1.0f), splat(-2.0f));                  // -d
+        const float2 ndl = fma2(e, splat(-1.0f), add2(d, splat(-2.0f)));        // -dl = (d - 2) - E
+        const float2 rc = rcp_2(d);
+        const float2 s0 = mul2(e, rc);
+        const float2 res = fma2(ndl, s0, fma2(nd, s0, e));
+        const float2 sq = fma2(res, rc, s0);
+        const float2 z = mul2(sq, sq);
+        float2 p = fma2(z, splat(0.12150468f), splat(0.10713829f));
+        p = fma2(p, z, splat(0.14308442f));
+        p = fma2(p, z, splat(0.19999439f));
+        p = fma2(p, z, splat(0.33333337f));
+        const float2 h = fma2(mul2(sq, z), p, sq);                               // atanh(s)
+        return fma2(h, splat(2.0f), relu2(x));
     } else if constexpr (ACT == FEWBIT_LEAKY_RELU) {
         const float2 m = mul2(x, splat(0.01f));
         return make_float2(fmaxf(x.x, m.x), fmaxf(x.y, m.y));
