@@ -127,6 +127,21 @@ def test_hot_path_argument_checks_need_no_gpu(lib):
     assert lib.fewbit_fwd_host(h, A, A, A, 10, 0, A, 16) == 5
     assert lib.fewbit_bwd_host(h, A, A, A, 10, 0, A + 8, 1 << 20) == 3
     assert lib.fewbit_fwd_host(h, A, A, A, 0, 0, None, 0) == 0
+    # f(x + bias): x, bias, y, packed, rows, cols
+    assert lib.fewbit_fwd_bias(None, A, A, A, A, 4, 1024, 1, None) == 1
+    assert lib.fewbit_fwd_bias(h, A, None, A, A, 4, 1024, 1, None) == 1
+    assert lib.fewbit_fwd_bias(h, A, A, A, A, 4, 1020, 1, None) == 2         # a row is not a whole number of 8-element chunks
+    assert lib.fewbit_fwd_bias(h, A, A, A, A, 4, 1 << 32, 1, None) == 2       # row length beyond 32 bits
+    assert lib.fewbit_fwd_bias(h, A, A + 16, A, A, 4, 1024, 1, None) == 3
+    assert lib.fewbit_fwd_bias(h, A, A, A, A, 1 << 40, 1 << 30, 1, None) == 1  # rows * cols overflows
+    assert lib.fewbit_fwd_bias(h, None, None, None, None, 0, 1024, 1, None) == 0
+    tf = fb.fewbit_table_create_folded("tanh", 2)
+    assert lib.fewbit_fwd_bias(tf.handle, A, A, A, A, 4, 1024, 1, None) == 2  # no folded tables with a bias
+    # the accuracy scan: act, first pattern, count, result
+    assert lib.fewbit_f32_activation_scan(99, 0, 16, A, None) == 1
+    assert lib.fewbit_f32_activation_scan(0, 0, 16, None, None) == 1
+    assert lib.fewbit_f32_activation_scan(0, 1 << 32, 1, A, None) == 1
+    assert lib.fewbit_f32_activation_scan(0, 0, 16, A + 4, None) == 3
 
 
 def test_host_workspace_bytes(lib):
