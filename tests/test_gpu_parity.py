@@ -247,6 +247,58 @@ def test_shards_cut_by_shard_range_concatenate_to_the_single_launch_stream():
             assert torch.equal(torch.cat(gis).view(torch.int16), gi.view(torch.int16))
 
 
+def _unpack_on_device(pk, bits, n):
+    w = pk.view(torch.int32).to(torch.int64) & 0xFFFFFFFF
+    pos = torch.arange(n, device=DEV, dtype=torch.int64) * bits
+    lo = w[pos >> 5] >> (pos & 31)
+    nxt = w[torch.clamp((pos >> 5) + 1, max=w.numel() - 1)] << (32 - (pos & 31))
+    return (lo | torch.where((pos & 31) + bits > 32, nxt, torch.zeros_like(lo))) & ((1 << bits) - 1)
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_randomised_tables_sizes_dtypes_under_every_variant(seed, monkeypatch):
+    """Random activation, bit width, dtype, size (ragged, whole warp-blocks, several waves), built-in
+    or injected tables (random boundaries, duplicates, tiny and large scales), inputs with zeros,
+    infinities, NaNs and subnormals: every bucketize variant (search, table with dynamic and with
+    static distribution, size-based choice) gives the same y and packed words, and the codes are
+    torch.bucketize's."""
+    import random
+    rng = random.Random(seed)
+    nprng = np.random.default_rng(seed)
+    acts = wl.ACTIVATIONS + wl.EXTRA_ACTIVATIONS
+    for _ in range(40):
+        dtype, act, bits = rng.choice(["f32", "bf16", "f16"]), rng.choice(acts), rng.randint(1, 4)
+        n = rng.choice([rng.randint(1, 5000), rng.randint(5000, 3_000_000), 1024 * rng.randint(1, 3000), (1 << 23) + rng.randint(0, 3000)])
+        if rng.random() < 0.5:
+            t = table(act, bits)
+        else:
+            s = np.sort(nprng.standard_normal((1 << bits) - 1).astype(np.float32) * np.float32(10.0 ** rng.uniform(-3, 1.5)))
+            if bits > 1 and rng.random() < 0.3:
+                s[rng.randrange(s.size - 1) + 1] = s[0]
+                s = np.sort(s)
+            t = fb.fewbit_table_from_arrays(act, bits, s, nprng.standard_normal(1 << bits).astype(np.float32))
+        x = (torch.randn(n, device=DEV) * 10.0 ** rng.uniform(-2, 1.3)).to(TORCH_DT[dtype])
+        if n > 10:
+            special = rng.choice([0.0, -0.0, float("inf"), float("-inf"), float("nan"), 1e-40, -1e-40, 65504.0, -3e38])
+            x[torch.randint(0, n, (min(n, 50),), device=DEV)] = torch.tensor(special, device=DEV).to(TORCH_DT[dtype])
+        s_np, _ = t.arrays()
+        want = torch.bucketize(x.float(), torch.from_numpy(np.ascontiguousarray(s_np)).to(DEV), right=False)
+        want = torch.where(torch.isnan(x.float()), torch.zeros_like(want), want)
+        outs = []
+        for mode, queue in (("never", None), ("always", None), ("always", "never"), ("auto", None)):
+            monkeypatch.setenv("FEWBIT_FWD_TABLE", mode)
+            if queue:
+                monkeypatch.setenv("FEWBIT_FWD_QUEUE", queue)
+            else:
+                monkeypatch.delenv("FEWBIT_FWD_QUEUE", raising=False)
+            outs.append(fb.fewbit_fwd(t, x))
+        torch.cuda.synchronize()
+        what = (seed, dtype, act, bits, n)
+        assert torch.equal(_unpack_on_device(outs[0][1], bits, n), want), what
+        for y, pk in outs[1:]:
+            assert torch.equal(pk, outs[0][1]) and torch.equal(y.view(torch.uint8), outs[0][0].view(torch.uint8)), what
+
+
 # --------------------------------------------------------------------------
 # bias in front of the activation
 # --------------------------------------------------------------------------
