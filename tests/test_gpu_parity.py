@@ -299,6 +299,38 @@ def test_randomised_tables_sizes_dtypes_under_every_variant(seed, monkeypatch):
             assert torch.equal(pk, outs[0][1]) and torch.equal(y.view(torch.uint8), outs[0][0].view(torch.uint8)), what
 
 
+@pytest.mark.parametrize("seed", [4, 5])
+def test_randomised_backward_and_bias_against_torch_arithmetic(seed, monkeypatch):
+    """Random sizes, dtypes, activations and bit widths: grad_in equals torch's binary32 product
+    rounded once, and f(x + bias) equals the plain forward on torch's binary32 sum rounded once."""
+    import random
+    rng = random.Random(seed)
+    for _ in range(40):
+        dtype, act, bits = rng.choice(["f32", "bf16", "f16"]), rng.choice(wl.ACTIVATIONS + wl.EXTRA_ACTIVATIONS), rng.randint(1, 4)
+        t = table(act, bits)
+        _, lev = t.arrays()
+        n = rng.choice([rng.randint(1, 5000), rng.randint(5000, 2_000_000), 1024 * rng.randint(1, 2000)])
+        x = (torch.randn(n, device=DEV) * 2).to(TORCH_DT[dtype])
+        g = (torch.randn(n, device=DEV) * 10.0 ** rng.uniform(-6, 3)).to(TORCH_DT[dtype])
+        _, pk = fb.fewbit_fwd(t, x)
+        gi = fb.fewbit_bwd(t, pk, g)
+        codes = _unpack_on_device(pk, bits, n)
+        want = (g.float() * torch.from_numpy(np.ascontiguousarray(lev)).to(DEV)[codes]).to(TORCH_DT[dtype])
+        assert torch.equal(gi.view(torch.uint8), want.view(torch.uint8)), (seed, dtype, act, bits, n)
+        cols = 8 * rng.randint(1, 1500)
+        rows = rng.randint(1, max(1, 400000 // cols))
+        xb = (torch.randn(rows, cols, device=DEV) * 2).to(TORCH_DT[dtype])
+        b = torch.randn(cols, device=DEV).to(TORCH_DT[dtype])
+        z = (xb.float() + b.float()[None, :]).to(TORCH_DT[dtype])
+        for mode in ("never", "always"):
+            monkeypatch.setenv("FEWBIT_FWD_TABLE", mode)
+            y1, p1 = fb.fewbit_fwd_bias(t, xb, b)
+            y2, p2 = fb.fewbit_fwd(t, z)
+            torch.cuda.synchronize()
+            assert torch.equal(p1, p2) and torch.equal(y1.view(torch.uint8), y2.view(torch.uint8)), (seed, dtype, act, bits, rows, cols, mode)
+        monkeypatch.delenv("FEWBIT_FWD_TABLE")
+
+
 # --------------------------------------------------------------------------
 # bias in front of the activation
 # --------------------------------------------------------------------------
