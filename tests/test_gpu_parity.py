@@ -808,6 +808,30 @@ def test_host_entry_points_match_the_oracle(dtype, pinned):
         compare_full("softplus", bits, x, g, y, p, gi, f"host {dtype} k={bits}")
 
 
+def test_host_entry_points_with_a_small_workspace_equal_the_device_path():
+    """A workspace much smaller than the tensor: every pipeline stage is reused several times, with
+    every bit width, and the bytes that come back must be those of the single device-resident launch."""
+    n = (1 << 23) + 4133
+    gen = torch.Generator().manual_seed(99)
+    x = torch.randn(n, generator=gen).to(torch.bfloat16).pin_memory()
+    g = torch.randn(n, generator=gen).to(torch.bfloat16).pin_memory()
+    for bits in (1, 2, 3, 4):
+        t = table("gelu", bits)
+        words = fb.fewbit_packed_bytes(n, bits) // 4
+        y = torch.empty(n, dtype=x.dtype).pin_memory()
+        gi = torch.empty(n, dtype=x.dtype).pin_memory()
+        p = torch.empty(words, dtype=torch.int32).pin_memory()
+        ws = torch.empty(fb.fewbit_host_workspace_bytes(1 << 20, x.dtype, bits), dtype=torch.uint8, device=DEV)
+        for _ in range(2):                     # the second pass finds the workspace dirty
+            y.fill_(3.0), gi.fill_(3.0), p.fill_(0x55555555)
+            fb.fewbit_fwd_host(t, x, y, p, ws)
+            fb.fewbit_bwd_host(t, p, g, gi, ws)
+            y_d, p_d, gi_d = run_gpu("gelu", bits, x.to(DEV), g.to(DEV))
+            assert torch.equal(p, p_d.cpu()), bits
+            assert torch.equal(y.view(torch.int16), y_d.cpu().view(torch.int16)), bits
+            assert torch.equal(gi.view(torch.int16), gi_d.cpu().view(torch.int16)), bits
+
+
 # --------------------------------------------------------------------------
 # ReLU / SELU and the autograd layer
 # --------------------------------------------------------------------------
