@@ -15,6 +15,7 @@ on the data path), time is the max over ranks.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import datetime
 import json
 import os
@@ -495,6 +496,49 @@ def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False, b
             "launches_per_timing": inner, "cases": out}
 
 
+def copy_at_size(nbytes: int, dev, reps: int = 10):
+    """GB/s of a torch copy_ that reads nbytes and writes nbytes, timed like quick_config (L2-cold by
+    rotation, short launches as a back-to-back batch): what a plain copy reaches at a given size."""
+    sets = max(2, (512 << 20) // (2 * nbytes) + 1)
+    inner = max(1, min(sets, (512 << 20) // (4 * nbytes)))
+    src = [torch.zeros(nbytes, dtype=torch.uint8, device=dev) for _ in range(sets)]
+    dst = [torch.empty(nbytes, dtype=torch.uint8, device=dev) for _ in range(sets)]
+    ms = []
+    for i in range(reps + 3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(400000)
+        e0.record()
+        for j in range(inner):
+            dst[(i * inner + j) % sets].copy_(src[(i * inner + j) % sets])
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            ms.append(e0.elapsed_time(e1) / inner)
+    return 2 * nbytes / (statistics.median(ms) * 1e-3) / 1e9
+
+
+def run_sweep(args):
+    """The size / activation / width / dtype sweep (config 5) at its points of at least 16 M elements:
+    one JSON line with the forward and backward time of every case and the fraction of the measured copy
+    bandwidth each reaches.  A context run on one GPU, not the contract line."""
+    import paper_2202_00441_b200 as fb
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peak()
+    out = {}
+    for case in wl.sweep_cases(tuple(n for n in wl.SWEEP_SIZES if n >= 1 << 24)):
+        if args.act:
+            case = dataclasses.replace(case, acts=(args.act,))
+        r = quick_config(fb, case, dev, reps=7)
+        for c in r["cases"].values():
+            c["fwd_frac"], c["bwd_frac"] = c["fwd_gbs"] / peak, c["bwd_gbs"] / peak
+        # a plain copy with the traffic of the 2-bit kernels of this size, for scale
+        r["torch_copy_same_traffic_frac"] = copy_at_size(int(algorithmic_bytes(case, case.n, 2)) // 2, dev) / peak
+        out[case.name] = r
+        torch.cuda.empty_cache()
+    print(json.dumps({"sweep": "c5, n >= 2^24", "peak_gbs": peak, "peak_kind": f"of {peak_kind}", "cases": out}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -512,7 +556,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-torch-baseline", action="store_true")
     ap.add_argument("--no-also", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time config 5 (7 activations x 1-4 bits x bf16/fp32 at 2^24, 2^24+7 and 2^28 elements) instead")
     args = ap.parse_args()
+    if args.sweep:
+        return run_sweep(args)
     args.warmup = max(args.warmup, 0)
     case = wl.CONFIGS[args.workload]
     act = args.act or case.acts[0]

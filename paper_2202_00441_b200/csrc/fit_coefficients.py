@@ -22,6 +22,10 @@ build or run time.
    degree 9 in u = w - 1/2, fitted on t in [0, 15] (w in [1/4, 1]) in the
    Chebyshev basis, relative error minimised; printed as monomials in u with
    the constant term split into a float32 value and the float32 remainder.
+
+4. Softplus for bfloat16 and binary16 storage.
+   log(1 + E) = E h(E), h(u) = log(1 + u) / u of degree 5 on u in [0, 1], relative
+   error minimised on Chebyshev nodes (8.4e-6).
 """
 import mpmath as mp
 import numpy as np
@@ -85,6 +89,25 @@ def fit_gelu_f32(p=0.2, deg=9, centre=0.5, tmax=15.0, nodes=500):
     return mono, err
 
 
+def fit_softplus_16(deg=5, nodes=600):
+    from numpy.polynomial import chebyshev as C, polynomial as P
+    k = np.arange(nodes)
+    z = np.cos(np.pi * (k + 0.5) / nodes)
+    u = (z + 1) / 2
+    target = np.array([float(mp.log1p(mp.mpf(v)) / mp.mpf(v)) for v in u])
+    V = C.chebvander(z, deg)
+    w = np.ones(nodes)
+    for _ in range(80):
+        c, *_ = np.linalg.lstsq(V * (w / target)[:, None], w, rcond=None)
+        err = (V @ c - target) / target
+        w = w * (1 + 4 * np.abs(err) / np.abs(err).max())
+        w /= w.mean()
+    mono = np.zeros(1)
+    for cf in C.cheb2poly(c)[::-1]:
+        mono = P.polyadd(P.polymul(mono, [-1.0, 2.0]), [cf])       # z = 2 u - 1
+    return mono, np.abs(err).max()
+
+
 if __name__ == "__main__":
     c, err = fit_gelu_log2()
     print("GELU bf16: L(16 s) coefficients (s^0..s^8):", ", ".join("%.9g" % np.float32(v) for v in c),
@@ -104,3 +127,6 @@ if __name__ == "__main__":
     bits = np.array([float(ln2)], dtype=np.float32).view(np.uint32) & np.uint32(0xfffffe00)
     hi = float(bits.view(np.float32)[0])
     print("ln 2 split: hi = %.15g, lo = %.15g" % (hi, float(ln2 - mp.mpf(hi))))
+    h, err = fit_softplus_16()
+    print("softplus 16-bit: h coefficients (u^0..u^5):", ", ".join("%.9g" % np.float32(v) for v in h),
+          "max relative error %.3e" % err)
