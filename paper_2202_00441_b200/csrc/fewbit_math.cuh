@@ -7,7 +7,7 @@
 // number of T (bfloat16 has the exponent range of binary32).
 //
 //   T = bfloat16 : binary32 arithmetic with hardware approximations (ex2, rcp,
-//                  lg2, tanh: relative error <= 2^-11, far below the 2^-9 that
+//                  tanh: relative error <= 2^-11, far below the 2^-9 that
 //                  one bfloat16 ulp allows).  Every form is written so that
 //                  the small quantity is computed as a product, never as a
 //                  difference of nearly equal numbers:
@@ -15,7 +15,7 @@
 //                      ex2.approx.ftz never flushes them) and the factor
 //                      2^-64 is folded into the last fused multiply-add, whose
 //                      IEEE gradual underflow gives correct subnormals.
-//   T = half     : as bfloat16 where the hardware approximation is 2^-22 (ex2, rcp, lg2), with a
+//   T = half     : as bfloat16 where the hardware approximation is 2^-22 (ex2, rcp), with a
 //                  tighter GELU fit (3.4e-5) and tanh / expm1 from ex2 instead of tanh.approx
 //                  (2^-11 is not enough for 11 significant bits).
 //   T = float    : binary32 arithmetic built on an exponential good to ~0.7 ulp, with the
@@ -37,11 +37,9 @@ namespace fewbit {
 // ---- hardware approximations ------------------------------------------------
 __device__ __forceinline__ float ex2_ftz(float a) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a)); return r; }
 __device__ __forceinline__ float rcp_ftz(float a) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a)); return r; }
-__device__ __forceinline__ float lg2_ftz(float a) { float r; asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a)); return r; }
 __device__ __forceinline__ float tanh_apx(float a) { float r; asm("tanh.approx.f32 %0, %1;" : "=f"(r) : "f"(a)); return r; }
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kScaleUp = 64.0f;                      // exponent offset S
 constexpr float kScaleDown = 5.421010862427522e-20f;   // 2^-64
 constexpr float kSeluScale = 1.0507009873554805f;       // lambda
@@ -372,7 +370,7 @@ __device__ __forceinline__ float2 act_f16(float2 x) {
     } else if constexpr (ACT == FEWBIT_ELU || ACT == FEWBIT_SELU) {
         return act_f32<ACT>(x);                     // exact-constant expm1, already good to 1-2 binary32 ulp
     } else {
-        return act_bf16<ACT>(x);                    // ex2 / rcp / lg2 forms: hardware error 2^-22
+        return act_bf16<ACT>(x);                    // ex2 / rcp forms: hardware error 2^-22
     }
 }
 
