@@ -448,6 +448,25 @@ def torch_unfused(case: wl.Case, act: str, x, g, reps: int = 5):
             "saved_bytes_per_elem": eb, "note": "stock torch forward + autograd backward, full input kept"}
 
 
+def batch_median_ms(launch, inner: int, reps: int) -> float:
+    """Median over `reps` timings (after 3 untimed ones) of a back-to-back batch of `inner` launches,
+    per launch, in ms: launch(i, j) enqueues launch j of timing i.  A spin kernel ahead of the first
+    event keeps the GPU busy (no memory traffic) while the host enqueues, so the events bracket GPU
+    time, not launch latency."""
+    ms = []
+    for i in range(reps + 3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(400000)
+        e0.record()
+        for j in range(inner):
+            launch(i, j)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            ms.append(e0.elapsed_time(e1) / inner)
+    return statistics.median(ms)
+
+
 def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False, bias_cols: int = 0):
     """Device-resident timing of another configuration.  L2-cold by rotation: enough independent
     buffer sets that their footprint exceeds 4x the 126 MB L2, a different set for every launch
@@ -460,7 +479,6 @@ def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False, b
     sets = max(2, int(512 * 2 ** 20 // per_set) + 1)
     # the event clock ticks every ~2 us: short kernels are timed as a back-to-back batch (launch gaps included)
     inner = max(1, min(sets, int(512 * 2 ** 20 // per_set)))
-    primed = False
     x0, g0 = wl.draw(case, dev)
     xs = [x0] + [x0.clone() for _ in range(sets - 1)]
     gs = [g0] + [g0.clone() for _ in range(sets - 1)]
@@ -474,56 +492,25 @@ def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False, b
         for b in case.bits:
             t = fb.fewbit_table_create_folded(act, b) if folded else fb.fewbit_table_create(act, b)
             ps = [torch.empty(fb.fewbit_packed_bytes(case.n, b) // 4, dtype=torch.int32, device=dev) for _ in range(sets)]
-            f_ms, b_ms = [], []
-            for i in range(reps + 3):
-                e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-                torch.cuda._sleep(400000)       # keeps the GPU busy (no memory traffic) while the host enqueues
-                e[0].record()
-                for j in range(inner):
-                    k = (i * inner + j) % sets
-                    if bias is None:
-                        fb.fewbit_fwd(t, xs[k], ys[k], ps[k])
-                    else:
-                        fb.fewbit_fwd_bias(t, xs[k].view(-1, bias_cols), bias, ys[k], ps[k])
-                e[1].record()
-                torch.cuda._sleep(400000)
-                e[2].record()
-                for j in range(inner):
-                    k = (i * inner + j) % sets
-                    fb.fewbit_bwd(t, ps[(k + 1) % sets] if primed else ps[k], gs[k], gis[k])
-                e[3].record()
-                torch.cuda.synchronize()
-                primed = True
-                if i >= 3:
-                    f_ms.append(e[0].elapsed_time(e[1]) / inner); b_ms.append(e[2].elapsed_time(e[3]) / inner)
+
+            def fwd(k):
+                if bias is None:
+                    fb.fewbit_fwd(t, xs[k], ys[k], ps[k])
+                else:
+                    fb.fewbit_fwd_bias(t, xs[k].view(-1, bias_cols), bias, ys[k], ps[k])
+
+            # cold: a different buffer set every launch (the forward timings leave codes in every set)
+            fm = batch_median_ms(lambda i, j: fwd((i * inner + j) % sets), inner, reps)
+            bm = batch_median_ms(lambda i, j: fb.fewbit_bwd(t, ps[(i * inner + j) % sets], gs[(i * inner + j) % sets],
+                                                            gis[(i * inner + j) % sets]), inner, reps)
             by = algorithmic_bytes(case, case.n, b)
-            fm, bm = statistics.median(f_ms), statistics.median(b_ms)
             out[f"{act}_k{b}"] = {"fwd_us": 1e3 * fm, "bwd_us": 1e3 * bm, "fwd_gbs": by / (fm * 1e-3) / 1e9,
                                   "bwd_gbs": by / (bm * 1e-3) / 1e9}
             if case.n * (2 * eb + 0.5) < 100 * 2 ** 20:
                 # L2-warm, labelled as such: the same buffers again and again (what one kernel touches fits the 126 MB L2)
                 warm = max(inner, 8)
-                w_ms = []
-                for i in range(reps + 3):
-                    e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-                    torch.cuda._sleep(400000)
-                    e[0].record()
-                    for j in range(warm):
-                        if bias is None:
-                            fb.fewbit_fwd(t, xs[0], ys[0], ps[0])
-                        else:
-                            fb.fewbit_fwd_bias(t, xs[0].view(-1, bias_cols), bias, ys[0], ps[0])
-                    e[1].record()
-                    torch.cuda._sleep(400000)
-                    e[2].record()
-                    for j in range(warm):
-                        fb.fewbit_bwd(t, ps[0], gs[0], gis[0])
-                    e[3].record()
-                    torch.cuda.synchronize()
-                    if i >= 3:
-                        w_ms.append((e[0].elapsed_time(e[1]) / warm, e[2].elapsed_time(e[3]) / warm))
-                out[f"{act}_k{b}"]["fwd_us_l2_warm"] = 1e3 * statistics.median(w[0] for w in w_ms)
-                out[f"{act}_k{b}"]["bwd_us_l2_warm"] = 1e3 * statistics.median(w[1] for w in w_ms)
+                out[f"{act}_k{b}"]["fwd_us_l2_warm"] = 1e3 * batch_median_ms(lambda i, j: fwd(0), warm, reps)
+                out[f"{act}_k{b}"]["bwd_us_l2_warm"] = 1e3 * batch_median_ms(lambda i, j: fb.fewbit_bwd(t, ps[0], gs[0], gis[0]), warm, reps)
     return {"workload": case.name, "elements": case.n, "dtype": case.dtype,
             "l2": f"cold by rotation over {sets} buffer sets ({sets * per_set / 2 ** 20:.0f} MiB)",
             "launches_per_timing": inner, "cases": out}
@@ -536,18 +523,8 @@ def copy_at_size(nbytes: int, dev, reps: int = 10):
     inner = max(1, min(sets, (512 << 20) // (4 * nbytes)))
     src = [torch.zeros(nbytes, dtype=torch.uint8, device=dev) for _ in range(sets)]
     dst = [torch.empty(nbytes, dtype=torch.uint8, device=dev) for _ in range(sets)]
-    ms = []
-    for i in range(reps + 3):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda._sleep(400000)
-        e0.record()
-        for j in range(inner):
-            dst[(i * inner + j) % sets].copy_(src[(i * inner + j) % sets])
-        e1.record()
-        torch.cuda.synchronize()
-        if i >= 3:
-            ms.append(e0.elapsed_time(e1) / inner)
-    return 2 * nbytes / (statistics.median(ms) * 1e-3) / 1e9
+    ms = batch_median_ms(lambda i, j: dst[(i * inner + j) % sets].copy_(src[(i * inner + j) % sets]), inner, reps)
+    return 2 * nbytes / (ms * 1e-3) / 1e9
 
 
 def run_sweep(args):
