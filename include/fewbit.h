@@ -109,7 +109,8 @@ FEWBIT_API fewbit_status fewbit_table_from_arrays(fewbit_act act, int bits, cons
 
 /*
  * Folded table for an activation whose derivative is even (caption of Fig. 3:
- * "we can quantize only positive real axis", which is worth one more bit):
+ * for such an f only the non-negative half-axis needs intervals, which is
+ * worth one more bit):
  * 2^bits pieces on [0, B], found by the same dynamic programme on a grid of
  * n_cells cells; the code of x is then #{ j : s[j] < |x| }.  Defined for
  * FEWBIT_SIGMOID and FEWBIT_TANH, otherwise FEWBIT_ERR_UNSUPPORTED.  The

@@ -163,7 +163,7 @@ std::shared_ptr<const Solved> solved_for(fewbit_act act, double A, double B, int
 }
 
 // ---------------------------------------------------------------------------
-// Off-grid refinement (Sec. 3: the DP result "can be finetuned using gradient-based methods").
+// Off-grid refinement (Sec. 3 proposes gradient-based fine-tuning of the grid optimum the DP returns).
 // ---------------------------------------------------------------------------
 struct BinSums { double w, fw, f2w; };
 
