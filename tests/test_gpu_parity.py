@@ -298,6 +298,43 @@ def test_randomised_tables_sizes_dtypes_under_every_variant(seed, monkeypatch):
             assert torch.equal(pk, outs[0][1]) and torch.equal(y.view(torch.uint8), outs[0][0].view(torch.uint8)), what
 
 
+@pytest.mark.parametrize("seed", [6, 7])
+def test_randomised_folded_tables_under_every_variant(seed, monkeypatch):
+    """Folded tables (caption of Fig. 3) with random range and grid, random dtype, size and input
+    scale: the codes are torch.bucketize's of |x| (NaN -> 0), the same under every bucketize variant,
+    and the backward product is torch's binary32 product rounded once."""
+    import random
+    rng = random.Random(seed)
+    for _ in range(30):
+        dtype, act, bits = rng.choice(["f32", "bf16", "f16"]), rng.choice(["sigmoid", "tanh"]), rng.randint(1, 4)
+        t = fb.fewbit_table_create_folded(act, bits, B=rng.uniform(2.0, 12.0), n_cells=rng.choice([64, 257, 1000, 2048, 4096]))
+        n = rng.choice([rng.randint(1, 5000), rng.randint(5000, 3_000_000), 1024 * rng.randint(1, 3000), (1 << 23) + rng.randint(0, 3000)])
+        x = (torch.randn(n, device=DEV) * 10.0 ** rng.uniform(-2, 1.3)).to(TORCH_DT[dtype])
+        if n > 10:
+            special = rng.choice([0.0, -0.0, float("inf"), float("-inf"), float("nan"), 1e-40, -1e-40, 65504.0, -3e38])
+            x[torch.randint(0, n, (min(n, 50),), device=DEV)] = torch.tensor(special, device=DEV).to(TORCH_DT[dtype])
+        g = torch.randn(n, device=DEV).to(TORCH_DT[dtype])
+        s_np, lev = t.arrays()
+        want = torch.bucketize(x.float().abs(), torch.from_numpy(np.ascontiguousarray(s_np)).to(DEV), right=False)
+        want = torch.where(torch.isnan(x.float()), torch.zeros_like(want), want)
+        outs = []
+        for mode, queue in (("never", None), ("always", None), ("always", "never"), ("auto", None)):
+            monkeypatch.setenv("FEWBIT_FWD_TABLE", mode)
+            if queue:
+                monkeypatch.setenv("FEWBIT_FWD_QUEUE", queue)
+            else:
+                monkeypatch.delenv("FEWBIT_FWD_QUEUE", raising=False)
+            outs.append(fb.fewbit_fwd(t, x))
+        torch.cuda.synchronize()
+        what = (seed, dtype, act, bits, n)
+        assert torch.equal(_unpack_on_device(outs[0][1], bits, n), want), what
+        for y, pk in outs[1:]:
+            assert torch.equal(pk, outs[0][1]) and torch.equal(y.view(torch.uint8), outs[0][0].view(torch.uint8)), what
+        gi = fb.fewbit_bwd(t, outs[0][1], g)
+        prod = (g.float() * torch.from_numpy(np.ascontiguousarray(lev)).to(DEV)[want]).to(TORCH_DT[dtype])
+        assert torch.equal(gi.view(torch.uint8), prod.view(torch.uint8)), what
+
+
 @pytest.mark.parametrize("seed", [4, 5])
 def test_randomised_backward_and_bias_against_torch_arithmetic(seed, monkeypatch):
     """Random sizes, dtypes, activations and bit widths: grad_in equals torch's binary32 product
