@@ -77,19 +77,19 @@ __device__ __forceinline__ float2 act_bf16(float2 x) {
         l = fma2(l, s, splat(-1.00036657f + 4.0f + kScaleUp));
         return fma2(mul2(s, ex2_2(l)), splat(-kScaleDown), relu);
     } else if constexpr (ACT == FEWBIT_SILU) {
-        // x sigmoid(x) = max(x,0) - |x| E / (1 + E)
-        const float2 relu = relu2(x);
-        const float2 t = abs2_from_relu(relu, x);
-        const float2 e = ex2_2(fma2(t, splat(-kLog2e), splat(kScaleUp)));
-        const float2 r = rcp_2(fma2(e, splat(kScaleDown), splat(1.0f)));
-        return fma2(mul2(mul2(t, e), r), splat(-kScaleDown), relu);
+        // x / (1 + e^{-x}) with e^{-x} carried as e^{-x} 2^-64 (finite down to x = -133, below the
+        // last x whose result is a bfloat16 subnormal; flushed to 0 where 1 + e^{-x} = 1 anyway), so
+        // that r = 2^64 sigmoid(x) is a normal number over that range.  sigmoid(x) = 2^-64 r is then
+        // formed first: it may be a binary32 subnormal (x < -87), but keeps at least 9 more bits than
+        // the bfloat16 product can hold, and a tiny x meets an exact 0.5.
+        const float2 e = ex2_2(fma2(x, splat(-kLog2e), splat(-kScaleUp)));
+        const float2 r = rcp_2(add2(e, splat(kScaleDown)));
+        return mul2(x, mul2(r, splat(kScaleDown)));
     } else if constexpr (ACT == FEWBIT_SIGMOID) {
-        // x >= 0: 1 - E/(1+E);  x < 0: E/(1+E)
-        const float2 step = make_float2(x.x >= 0.0f ? 1.0f : 0.0f, x.y >= 0.0f ? 1.0f : 0.0f);
-        const float2 e = ex2_2(make_float2(fmaf(fabsf(x.x), -kLog2e, kScaleUp), fmaf(fabsf(x.y), -kLog2e, kScaleUp)));
-        const float2 q = mul2(e, rcp_2(fma2(e, splat(kScaleDown), splat(1.0f))));
-        const float2 sgn = fma2(step, splat(-2.0f), splat(1.0f));
-        return fma2(mul2(q, sgn), splat(kScaleDown), step);
+        // 1 / (1 + e^{-x}), same scaling: 2^-64 r
+        const float2 e = ex2_2(fma2(x, splat(-kLog2e), splat(-kScaleUp)));
+        const float2 r = rcp_2(add2(e, splat(kScaleDown)));
+        return mul2(r, splat(kScaleDown));
     } else if constexpr (ACT == FEWBIT_TANH) {
         return make_float2(tanh_apx(x.x), tanh_apx(x.y));
     } else if constexpr (ACT == FEWBIT_ELU) {
