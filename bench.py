@@ -204,9 +204,14 @@ def cpu_baseline(case: wl.Case, act: str, sample_elems: int):
     tables = oracle_tables(case, act)
     secs = oracle_pass(case, act, x_np, g_np, tables, threads)
     passes = 2 * len(case.bits) * sample_elems
+    # the same on one thread, on 1/16 of the sample (the oracle itself is single-threaded plain C)
+    one = max(1024, sample_elems // 16)
+    secs_one = oracle_pass(case, act, x_np[:one], g_np[:one], tables, 1)
     return {"value": passes / secs, "unit": "elements/s", "cores": threads, "kind": "oracle",
             "sample": f"first {sample_elems} elements of the {case.name} draw, bits {list(case.bits)}, fwd+bwd, "
-                      f"{threads} shards on {threads} threads, {secs:.2f} s"}
+                      f"{threads} shards on {threads} threads, {secs:.2f} s",
+            "value_one_thread": 2 * len(case.bits) * one / secs_one,
+            "sample_one_thread": f"first {one} elements, 1 thread, {secs_one:.2f} s"}
 
 
 # ----------------------------------------------------------------------------
