@@ -640,7 +640,7 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     // the previous kernel left idle, and a sub-wave grid then runs on part of the SMs (binary32
     // GELU, 2^20 elements: 8.3 -> 9.2 us).
     const bool issue_bound = sizeof(T) == 4 && act_weight(ACT) == 2;
-    const bool pdl = pdl_enabled() && grid >= static_cast<unsigned>(issue_bound ? slots : static_cast<size_t>(sms));
+    const bool pdl = pdl_enabled() && (!issue_bound || grid <= static_cast<unsigned>(sms) || grid >= static_cast<unsigned>(slots));
     return launch_pdl(kernel, grid, static_cast<unsigned>(warps_per_cta * 32), smem * warps_per_cta / (kFwdThreads / 32), st, pdl,
                       p2, static_cast<const T *>(x), static_cast<T *>(y), packed, n, static_cast<int>(iters), n_long);
 }

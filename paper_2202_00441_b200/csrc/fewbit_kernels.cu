@@ -168,20 +168,32 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
     if (sm_err != cudaSuccess) { t_last_cuda_error = static_cast<int>(sm_err); return FEWBIT_ERR_CUDA; }
     const size_t warps_per_cta = static_cast<size_t>(bf16 ? FwdThreads<__nv_bfloat16, true>::value : FwdThreads<float, true>::value) / 32;
     const size_t waves = n / kWarpElems / (warps_per_cta * slots);
-    // 16-bit types (measured at 2^24 .. 2^28 elements, dynamic distribution): the table wins from ~6
-    // waves at 4 bits, from ~20 at 3 bits (the packed search costs 3 comparisons there, 4 levels of
-    // selects at 4 bits)
-    bool use_lut = prm.runs.count != 0 && ((table->bits == 4 && waves >= 6) || (table->bits == 3 && waves >= 20));
+    // 16-bit types: from how many waves on the 64 KB pattern table beats the packed search, measured
+    // L2-cold at 2^24 .. 2^28 elements (3 .. 55 waves) for every activation, with dynamic distribution;
+    // 0 = never.  The heavier the arithmetic of f, the earlier the table's shorter instruction stream
+    // pays for its expansion and its bank conflicts; for the cheapest ones the search is faster at any size.
+    //                                             gelu silu sigm tanh elu  sopl leak relu selu
+    static const unsigned char kMinWavesBf16[2][FEWBIT_NUM_ACTS] = {{20,  0,   0,   0,   0,  20,  0,   0,   0},     // 3 bits
+                                                                    { 6, 12,  24,   0,  12,   6, 24,   0,   6}};    // 4 bits
+    static const unsigned char kMinWavesF16[2][FEWBIT_NUM_ACTS] = {{ 0,  0,   0,  24,  12,  48,  0,   0,  12},
+                                                                   {12, 24,   0,  12,   6,  12,  0,   0,   6}};
+    bool use_lut = false;
+    if (bf16 && prm.runs.count != 0 && table->bits >= 3) {
+        const unsigned min_waves = (dtype == FEWBIT_F16 ? kMinWavesF16 : kMinWavesBf16)[table->bits - 3][table->act];
+        use_lut = min_waves != 0 && waves >= min_waves;
+    }
     if (!bf16 && prm.runs.count != 0) {
-        // binary32 (measured, 2^22 .. 2^27 elements): at 4 bits the table beats the 4-level search at
-        // every size; at 3 bits only on large inputs, and for the light activations never
+        // binary32 (measured L2-cold at 2^20 .. 2^28 elements against the select-tree search): the 8 KB
+        // table wins at 4 bits from 2 waves for the lightest activations, from 4 for the others (8 for
+        // GELU, whose arithmetic hides the search longest); at 3 bits from 16 waves, never for ReLU-like
         const int weight = act_weight(table->act);
-        use_lut = table->bits == 4 || (table->bits == 3 && ((weight == 2 && waves >= kLutMinIters) || (weight == 1 && waves >= 24)));
+        const size_t min_waves4 = weight == 0 ? 2 : (table->act == FEWBIT_GELU ? 8 : 4);
+        use_lut = (table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && weight >= 1 && waves >= 16);
     }
     bool forced_table = false;
     if (const char *force = getenv("FEWBIT_FWD_TABLE")) {               // testing aid, see fewbit.h
-        if (force[0] == 'a') { use_lut = prm.runs.count != 0; forced_table = true; }   // "always"
-        else if (force[0] == 'n') use_lut = false;                        // "never"
+        if (force[0] == 'a' && force[1] == 'l') { use_lut = prm.runs.count != 0; forced_table = true; }   // "always"
+        else if (force[0] == 'n') use_lut = false;                        // "never"; anything else ("auto"): the size-based choice
     }
     // The table variants distribute their warp-blocks dynamically when a set of work counters can
     // be leased (not during stream capture); the 16-bit types at 3 bits only beat the packed search
