@@ -175,7 +175,7 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
     //                                             gelu silu sigm tanh elu  sopl leak relu selu
     static const unsigned char kMinWavesBf16[2][FEWBIT_NUM_ACTS] = {{20,  0,   0,   0,   0,  20,  0,   0,   0},     // 3 bits
                                                                     { 6, 12,  24,   0,  12,   6, 24,   0,   6}};    // 4 bits
-    static const unsigned char kMinWavesF16[2][FEWBIT_NUM_ACTS] = {{ 0,  0,   0,  24,  12,  48,  0,   0,  12},
+    static const unsigned char kMinWavesF16[2][FEWBIT_NUM_ACTS] = {{ 0,  0,   0,   0,  24,  48,  0,   0,  12},
                                                                    {12, 24,   0,  12,   6,  12,  0,   0,   6}};
     bool use_lut = false;
     if (bf16 && prm.runs.count != 0 && table->bits >= 3) {

@@ -16,8 +16,8 @@
 //                      2^-64 is folded into the last fused multiply-add, whose
 //                      IEEE gradual underflow gives correct subnormals.
 //   T = half     : as bfloat16 where the hardware approximation is 2^-22 (ex2, rcp), with a
-//                  tighter GELU fit (3.4e-5) and tanh / expm1 from ex2 instead of tanh.approx
-//                  (2^-11 is not enough for 11 significant bits).
+//                  tighter GELU fit (3.4e-5) and tanh / expm1 from ex2 and a short series near 0
+//                  instead of tanh.approx (2^-11 is not enough for 11 significant bits).
 //   T = float    : binary32 arithmetic built on an exponential good to ~0.7 ulp, with the
 //                  rounding error of every step that would reach the result carried along as a
 //                  second binary32 term (fused multiply-add residuals).  GELU against the
@@ -358,17 +358,26 @@ __device__ __forceinline__ float2 act_f16(float2 x) {
         l = fma2(l, s, splat(-1.00004601f + 2.5849625f + kScaleUp));
         return fma2(mul2(s, ex2_2(l)), splat(-kScaleDown), relu);
     } else if constexpr (ACT == FEWBIT_TANH) {
-        // |x| >= 1/32: (1 - E) / (1 + E), E = e^{-2|x|} (1 - E >= 0.06, no harmful cancellation);
-        // below: x - x^3/3 (relative error 2 x^4 / 15 < 2e-7)
-        const float2 relu = relu2(x);
-        const float2 t = abs2_from_relu(relu, x);
-        const float2 e = ex2_2(mul2(t, splat(-2.0f * kLog2e)));
-        const float2 big = mul2(fma2(e, splat(-1.0f), splat(1.0f)), rcp_2(add2(e, splat(1.0f))));
+        // |x| >= 1/32: 2 / (1 + E) - 1 with E = e^{-2x} for the signed x (E = inf gives -1, E = 0
+        // gives 1; the difference keeps 2^-16 relative accuracy down to 1/32); below: x - x^3/3
+        // (relative error 2 x^4 / 15 < 2e-7)
+        const float2 e = ex2_2(mul2(x, splat(-2.0f * kLog2e)));
+        const float2 big = fma2(rcp_2(add2(e, splat(1.0f))), splat(2.0f), splat(-1.0f));
         const float2 x2 = mul2(x, x);
         const float2 small = fma2(mul2(x2, x), splat(-0.33333334f), x);
-        return make_float2(t.x < 0.03125f ? small.x : copysignf(big.x, x.x), t.y < 0.03125f ? small.y : copysignf(big.y, x.y));
+        return make_float2(fabsf(x.x) < 0.03125f ? small.x : big.x, fabsf(x.y) < 0.03125f ? small.y : big.y);
     } else if constexpr (ACT == FEWBIT_ELU || ACT == FEWBIT_SELU) {
-        return act_f32<ACT>(x);                     // exact-constant expm1, already good to 1-2 binary32 ulp
+        // e^x - 1 for x <= 0 to binary16 accuracy: e^x - 1 by the hardware exponential below -1/32
+        // (the difference keeps 2^-17 there), x (1 + x/2 + x^2/6) above (next term x^3/24: 1.3e-6)
+        const float2 big = add2(ex2_2(mul2(x, splat(kLog2e))), splat(-1.0f));
+        const float2 small = mul2(x, fma2(x, fma2(x, splat(0.16666667f), splat(0.5f)), splat(1.0f)));
+        float2 m = make_float2(x.x < -0.03125f ? big.x : small.x, x.y < -0.03125f ? big.y : small.y);
+        float2 p = x;
+        if constexpr (ACT == FEWBIT_SELU) {
+            m = mul2(m, splat(kSeluScaleAlpha));
+            p = mul2(x, splat(kSeluScale));
+        }
+        return make_float2(x.x > 0.0f ? p.x : m.x, x.y > 0.0f ? p.y : m.y);
     } else {
         return act_bf16<ACT>(x);                    // ex2 / rcp forms: hardware error 2^-22
     }
