@@ -185,10 +185,12 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
     if (!bf16 && prm.runs.count != 0) {
         // binary32 (measured L2-cold at 2^20 .. 2^28 elements against the select-tree search): the 8 KB
         // table wins at 4 bits from 2 waves for the lightest activations, from 4 for the others (8 for
-        // GELU, whose arithmetic hides the search longest); at 3 bits from 16 waves, never for ReLU-like
+        // GELU, whose arithmetic hides the search longest); at 3 bits from 16 waves (4 for ELU and SELU),
+        // never for ReLU-like
         const int weight = act_weight(table->act);
         const size_t min_waves4 = weight == 0 ? 2 : (table->act == FEWBIT_GELU ? 8 : 4);
-        use_lut = (table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && weight >= 1 && waves >= 16);
+        const size_t min_waves3 = (table->act == FEWBIT_ELU || table->act == FEWBIT_SELU) ? 4 : 16;
+        use_lut = (table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && weight >= 1 && waves >= min_waves3);
     }
     bool forced_table = false;
     if (const char *force = getenv("FEWBIT_FWD_TABLE")) {               // testing aid, see fewbit.h
