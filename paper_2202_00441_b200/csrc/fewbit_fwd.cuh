@@ -495,17 +495,32 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         uint32_t w[BITS + 1];
 #pragma unroll
         for (int j = 0; j <= BITS; ++j) w[j] = 0;
+        // eight loads at a time ahead of their stores: y may alias x, so the compiler cannot move a load
+        // above a store, and 32 load-use-store rounds in a row would each pay the full memory latency
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            if (base + e < n) {
-                float xv = load1(x + base + e);
-                if constexpr (BIAS)                                  // the sum rounded once to the storage type
-                    xv = round_to<T>(__fadd_rn(xv, load1(static_cast<const T *>(prm.bias) + (base + e) % prm.cols)));
-                store1(y + base + e, activation<ACT, T>(xv));
-                const uint32_t c = bucketize<BITS>(prm.tb, FOLD ? fabsf(xv) : xv);
-                const int pos = e * BITS;
-                w[pos >> 5] |= c << (pos & 31);
-                if ((pos & 31) + BITS > 32) w[(pos >> 5) + 1] |= c >> (32 - (pos & 31));
+        for (int e0 = 0; e0 < 32; e0 += 8) {
+            float xs[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int e = e0 + i;
+                xs[i] = 0.0f;
+                if (base + e < n) {
+                    xs[i] = load1(x + base + e);
+                    if constexpr (BIAS)                              // the sum rounded once to the storage type
+                        xs[i] = round_to<T>(__fadd_rn(xs[i], load1(static_cast<const T *>(prm.bias) + (base + e) % prm.cols)));
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int e = e0 + i;
+                if (base + e < n) {
+                    const float xv = xs[i];
+                    store1(y + base + e, activation<ACT, T>(xv));
+                    const uint32_t c = bucketize<BITS>(prm.tb, FOLD ? fabsf(xv) : xv);
+                    const int pos = e * BITS;
+                    w[pos >> 5] |= c << (pos & 31);
+                    if ((pos & 31) + BITS > 32) w[(pos >> 5) + 1] |= c >> (32 - (pos & 31));
+                }
             }
         }
         const size_t total_words = (n * BITS + 31) / 32;
