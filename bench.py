@@ -482,8 +482,11 @@ def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False, b
     eb = elem_size(case)
     per_set = case.n * (4 * eb + 0.5)
     sets = max(2, int(512 * 2 ** 20 // per_set) + 1)
-    # the event clock ticks every ~2 us: short kernels are timed as a back-to-back batch (launch gaps included)
-    inner = max(1, min(sets, int(512 * 2 ** 20 // per_set)))
+    if per_set < 512 * 2 ** 20:
+        sets = max(sets, 9)
+    # the event clock ticks every ~2 us: short kernels are timed as a back-to-back batch of up to 8
+    # launches (launch gaps included), each on another buffer set
+    inner = max(1, min(sets - 1, 8)) if per_set < 512 * 2 ** 20 else 1
     x0, g0 = wl.draw(case, dev)
     xs = [x0] + [x0.clone() for _ in range(sets - 1)]
     gs = [g0] + [g0.clone() for _ in range(sets - 1)]
@@ -525,7 +528,9 @@ def copy_at_size(nbytes: int, dev, reps: int = 10):
     """GB/s of a torch copy_ that reads nbytes and writes nbytes, timed like quick_config (L2-cold by
     rotation, short launches as a back-to-back batch): what a plain copy reaches at a given size."""
     sets = max(2, (512 << 20) // (2 * nbytes) + 1)
-    inner = max(1, min(sets, (512 << 20) // (4 * nbytes)))
+    if 4 * nbytes < (512 << 20):
+        sets = max(sets, 9)
+    inner = max(1, min(sets - 1, 8)) if 4 * nbytes < (512 << 20) else 1
     src = [torch.zeros(nbytes, dtype=torch.uint8, device=dev) for _ in range(sets)]
     dst = [torch.empty(nbytes, dtype=torch.uint8, device=dev) for _ in range(sets)]
     ms = batch_median_ms(lambda i, j: dst[(i * inner + j) % sets].copy_(src[(i * inner + j) % sets]), inner, reps)
