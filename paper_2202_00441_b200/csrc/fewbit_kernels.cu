@@ -174,9 +174,9 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
     // pays for its expansion and its bank conflicts; for the cheapest ones the search is faster at any size.
     //                                             gelu silu sigm tanh elu  sopl leak relu selu
     static const unsigned char kMinWavesBf16[2][FEWBIT_NUM_ACTS] = {{20,  0,   0,   0,   0,  20,  0,   0,   0},     // 3 bits
-                                                                    { 6, 12,  24,   0,  12,   6, 24,   0,   6}};    // 4 bits
-    static const unsigned char kMinWavesF16[2][FEWBIT_NUM_ACTS] = {{ 0,  0,   0,   0,  24,  48,  0,   0,  12},
-                                                                   {12, 24,   0,  12,   6,  12,  0,   0,   6}};
+                                                                    { 3,  6,  24,   0,   6,   6, 24,   0,   6}};    // 4 bits
+    static const unsigned char kMinWavesF16[2][FEWBIT_NUM_ACTS] = {{ 0,  0,   0,   0,  24,  48,  0,   0,   6},
+                                                                   { 6, 24,   0,   6,   6,   6,  0,   0,   3}};
     bool use_lut = false;
     if (bf16 && prm.runs.count != 0 && table->bits >= 3) {
         const unsigned min_waves = (dtype == FEWBIT_F16 ? kMinWavesF16 : kMinWavesBf16)[table->bits - 3][table->act];
@@ -185,11 +185,11 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
     if (!bf16 && prm.runs.count != 0) {
         // binary32 (measured L2-cold at 2^20 .. 2^28 elements against the select-tree search): the 8 KB
         // table wins at 4 bits from 2 waves for the lightest activations, from 4 for the others (8 for
-        // GELU, whose arithmetic hides the search longest); at 3 bits from 16 waves (4 for ELU and SELU),
+        // GELU, whose arithmetic hides the search longest); at 3 bits from 16 waves (8 for ELU and SELU),
         // never for ReLU-like
         const int weight = act_weight(table->act);
         const size_t min_waves4 = weight == 0 ? 2 : (table->act == FEWBIT_GELU ? 8 : 4);
-        const size_t min_waves3 = (table->act == FEWBIT_ELU || table->act == FEWBIT_SELU) ? 4 : 16;
+        const size_t min_waves3 = (table->act == FEWBIT_ELU || table->act == FEWBIT_SELU) ? 8 : 16;
         use_lut = (table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && weight >= 1 && waves >= min_waves3);
     }
     bool forced_table = false;
