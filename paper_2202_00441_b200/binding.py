@@ -207,10 +207,38 @@ def fewbit_f32_activation_scan(act, first_pattern: int = 0, count: int = 1 << 32
     return {"hist": v[:4], "max_ulp": v[4] >> 32, "worst_pattern": v[4] & 0xFFFFFFFF}
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)    # the current stream's handle without building a Stream object
+
+
 def _stream_ptr(stream: Optional[torch.cuda.Stream], device) -> int:
-    if stream is None:
-        stream = torch.cuda.current_stream(device)
-    return stream.cuda_stream
+    if stream is not None:
+        return stream.cuda_stream
+    if _raw_stream is not None and device.index is not None:
+        return _raw_stream(device.index)
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+class _NoSwitch:
+    def __enter__(self):
+        return None
+
+    def __exit__(self, *exc):
+        return False
+
+
+_NO_SWITCH = _NoSwitch()
+
+
+def _current(device):
+    """Context that makes `device` current for the call; free when it already is (a launch on a
+    small tensor costs less than torch.cuda.device's own bookkeeping)."""
+    if device.index is None or device.index == torch.cuda.current_device():
+        return _NO_SWITCH
+    return torch.cuda.device(device)
+
+
+def _packed_bytes(n: int, bits: int) -> int:
+    return 4 * ((n * bits + 31) // 32)          # fewbit_packed_bytes without the foreign call
 
 
 def _dev_tensor(t: torch.Tensor, name: str) -> torch.Tensor:
@@ -229,11 +257,11 @@ def fewbit_fwd(table: Table, x: torch.Tensor, y: Optional[torch.Tensor] = None,
     if y is None:
         y = torch.empty_like(x)
     if packed is None:
-        packed = torch.empty(fewbit_packed_bytes(n, table.bits) // 4, dtype=torch.int32, device=x.device)
+        packed = torch.empty(_packed_bytes(n, table.bits) // 4, dtype=torch.int32, device=x.device)
     _dev_tensor(y, "y"), _dev_tensor(packed, "packed")
-    if y.dtype != x.dtype or y.numel() != n or packed.numel() * packed.element_size() < fewbit_packed_bytes(n, table.bits):
+    if y.dtype != x.dtype or y.numel() != n or packed.numel() * packed.element_size() < _packed_bytes(n, table.bits):
         raise ValueError("y / packed do not match x")
-    with torch.cuda.device(x.device):
+    with _current(x.device):
         _check(lib.fewbit_fwd(table.handle, x.data_ptr(), y.data_ptr(), packed.data_ptr(), n, _DTYPES[x.dtype],
                               _stream_ptr(stream, x.device)), "fewbit_fwd")
     return y, packed
@@ -253,11 +281,11 @@ def fewbit_fwd_bias(table: Table, x: torch.Tensor, bias: torch.Tensor, y: Option
     if y is None:
         y = torch.empty_like(x)
     if packed is None:
-        packed = torch.empty(fewbit_packed_bytes(n, table.bits) // 4, dtype=torch.int32, device=x.device)
+        packed = torch.empty(_packed_bytes(n, table.bits) // 4, dtype=torch.int32, device=x.device)
     _dev_tensor(y, "y"), _dev_tensor(packed, "packed")
-    if y.dtype != x.dtype or y.numel() != n or packed.numel() * packed.element_size() < fewbit_packed_bytes(n, table.bits):
+    if y.dtype != x.dtype or y.numel() != n or packed.numel() * packed.element_size() < _packed_bytes(n, table.bits):
         raise ValueError("y / packed do not match x")
-    with torch.cuda.device(x.device):
+    with _current(x.device):
         _check(lib.fewbit_fwd_bias(table.handle, x.data_ptr(), bias.data_ptr(), y.data_ptr(), packed.data_ptr(), rows, cols,
                                    _DTYPES[x.dtype], _stream_ptr(stream, x.device)), "fewbit_fwd_bias")
     return y, packed
@@ -273,9 +301,9 @@ def fewbit_bwd(table: Table, packed: torch.Tensor, grad_out: torch.Tensor,
         grad_in = torch.empty_like(grad_out)
     _dev_tensor(grad_in, "grad_in")
     if grad_in.dtype != grad_out.dtype or grad_in.numel() != n or \
-            packed.numel() * packed.element_size() < fewbit_packed_bytes(n, table.bits):
+            packed.numel() * packed.element_size() < _packed_bytes(n, table.bits):
         raise ValueError("grad_in / packed do not match grad_out")
-    with torch.cuda.device(grad_out.device):
+    with _current(grad_out.device):
         _check(lib.fewbit_bwd(table.handle, packed.data_ptr(), grad_out.data_ptr(), grad_in.data_ptr(), n,
                               _DTYPES[grad_out.dtype], _stream_ptr(stream, grad_out.device)), "fewbit_bwd")
     return grad_in
