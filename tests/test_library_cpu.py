@@ -41,6 +41,10 @@ def test_packed_bytes(lib):
         for n in (0, 1, 31, 32, 33, 1000, 2 ** 24 + 7, 2 ** 28):
             assert fb.fewbit_packed_bytes(n, bits) == 4 * ((n * bits + 31) // 32)
     assert fb.fewbit_packed_bytes(100, 0) == 0 and fb.fewbit_packed_bytes(100, 5) == 0
+    # the binding sizes its buffers without the foreign call: same numbers
+    for n in (0, 1, 31, 32, 33, 1023, 1025, 2 ** 24 + 7, 2 ** 33 + 5):
+        for bits in (1, 2, 3, 4):
+            assert fb.binding._packed_bytes(n, bits) == fb.fewbit_packed_bytes(n, bits)
 
 
 @pytest.mark.parametrize("act", ACTIVATIONS + EXTRA_ACTIVATIONS)
