@@ -185,10 +185,11 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  * Errors: FEWBIT_ERR_INVALID_ARG (NULL table or buffer, bad dtype),
  * FEWBIT_ERR_ALIGNMENT, FEWBIT_ERR_CUDA (launch failed).
  * The interval search has several equivalent kernel variants (binary search,
- * two-at-a-time bfloat16 search, shared-memory code table) chosen from bits,
- * dtype and n; all give identical codes.  The code-table variants (16-bit types
- * at 3-4 bits on large inputs, binary32 at 3-4 bits) distribute their work
- * through a set of counters in a
+ * two-at-a-time bfloat16 search, shared-memory code table) chosen from the
+ * activation, bits, dtype and n by measured thresholds; all give identical
+ * codes.  The code-table variants (3-4 bits, from a few waves of resident warps
+ * on, earlier the costlier f is) distribute their work through a set of
+ * counters in a
  * file-scope device array (16 sets per device; nothing is allocated, but the
  * first such call on a device creates up to 16 CUDA events, and each call
  * records one after its kernel).  While `stream` is being captured,
