@@ -176,7 +176,7 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  * Forward half, one kernel launch on `stream` (a cudaStream_t passed as
  * void*; NULL = the legacy default stream), asynchronous:
  *     y[e]      = f(x[e])                 exact activation, rounded to dtype
- *     code[e]   = #{ j : s[j] < x[e] }    Eq. 2 / "sortedsearch" of Listing 1
+ *     code[e]   = #{ j : s[j] < x[e] }    Eq. 2 / the sorted search of Listing 1
  *     packed    = the codes as a `bits`-bit stream (layout above)
  * x, y: DEVICE, n elements of `dtype`, 32-byte aligned; y == x (exact alias)
  * is allowed, any other overlap is undefined.  packed: DEVICE,
