@@ -130,7 +130,7 @@ __device__ __forceinline__ void store1(float *p, float v) { *p = v; }
 __device__ __forceinline__ void store1(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
 
 // ---------------------------------------------------------------------------
-// Eq. 2 / "sortedsearch": code = #{ j : s[j] < x }, a branch-free binary
+// Eq. 2 / the sorted search of Listing 1: code = #{ j : s[j] < x }, a branch-free binary
 // search over the 2^BITS - 1 sorted boundaries.  Every comparison is
 // `s < x` in binary32, so NaN compares false everywhere (code 0).
 // ---------------------------------------------------------------------------

@@ -91,7 +91,7 @@ def test_bf16_rounding_is_identity_on_bf16_values():
 
 
 # --------------------------------------------------------------------------
-# bucketize (Eq. 2 / "sortedsearch" of Listing 1)
+# bucketize (Eq. 2 / the sorted search of Listing 1)
 # --------------------------------------------------------------------------
 @pytest.mark.parametrize("bits", [1, 2, 3, 4])
 def test_bucketize_equals_searchsorted_left(bits):
