@@ -298,6 +298,40 @@ def test_randomised_tables_sizes_dtypes_under_every_variant(seed, monkeypatch):
             assert torch.equal(pk, outs[0][1]) and torch.equal(y.view(torch.uint8), outs[0][0].view(torch.uint8)), what
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_degenerate_boundary_tables(dtype, monkeypatch):
+    """Injected tables at the edges of what Eq. 2 allows: all boundaries equal, infinite boundaries,
+    boundaries at the smallest subnormal, at +-0 and beyond the binary16 range; inputs with zeros,
+    infinities, NaN, subnormals and the largest finite values.  Codes are torch.bucketize's under
+    every bucketize variant."""
+    inf = float("inf")
+    cases = {1: [[0], [inf], [-inf], [1e-45], [-1e-45], [65520], [3.4e38]],
+             2: [[0, 0, 0], [-inf, 0, inf], [-inf, -inf, -inf], [inf, inf, inf], [-3e38, 0, 3e38], [1e-45, 1e-45, 2e-45],
+                 [-0.0, 0.0, 0.0], [65504, 65504, 65520]],
+             3: [[-inf, -1, -1, 0, 1, 1, inf], [1e30] * 7],
+             4: [[-inf] * 5 + [0] * 5 + [inf] * 5, list(np.linspace(-1e-44, 1e-44, 15)), [7] * 15]}
+    special = [0.0, -0.0, inf, -inf, float("nan"), 1e-45, -1e-45, 1e-40, -1e-40, 6e-8, -6e-8, 65504.0, -65504.0, 65520.0,
+               3.3e38, -3.3e38, 7.0, 1.0, -1.0]
+    for bits, tables in cases.items():
+        for s in tables:
+            t = fb.fewbit_table_from_arrays("tanh", bits, np.array(s, dtype=np.float32), np.arange(1 << bits, dtype=np.float32))
+            s_np, _ = t.arrays()
+            edges = torch.from_numpy(np.ascontiguousarray(s_np)).to(DEV)
+            for n in (70000, (1 << 23) + 5):
+                x = (torch.randn(n, device=DEV) * 3).to(TORCH_DT[dtype])
+                x[:len(special)] = torch.tensor(special, device=DEV).to(TORCH_DT[dtype])
+                want = torch.bucketize(x.float(), edges, right=False)
+                want = torch.where(torch.isnan(x.float()), torch.zeros_like(want), want)
+                for mode, queue in (("never", None), ("always", None), ("always", "never")):
+                    monkeypatch.setenv("FEWBIT_FWD_TABLE", mode)
+                    if queue:
+                        monkeypatch.setenv("FEWBIT_FWD_QUEUE", queue)
+                    else:
+                        monkeypatch.delenv("FEWBIT_FWD_QUEUE", raising=False)
+                    _, pk = fb.fewbit_fwd(t, x)
+                    assert torch.equal(_unpack_on_device(pk, bits, n), want), (dtype, bits, s, n, mode, queue)
+
+
 @pytest.mark.parametrize("seed", [6, 7])
 def test_randomised_folded_tables_under_every_variant(seed, monkeypatch):
     """Folded tables (caption of Fig. 3) with random range and grid, random dtype, size and input
