@@ -332,6 +332,32 @@ def test_degenerate_boundary_tables(dtype, monkeypatch):
                     assert torch.equal(_unpack_on_device(pk, bits, n), want), (dtype, bits, s, n, mode, queue)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+def test_backward_with_special_levels_and_gradients(dtype):
+    """Levels and incoming gradients at the edges of the arithmetic (infinities, NaN, signed zeros,
+    subnormals, the largest finite values): grad_in is torch's binary32 product rounded once -- the
+    same bits wherever that is a number, NaN where it is NaN."""
+    inf, nan = float("inf"), float("nan")
+    lev = np.array([inf, -inf, nan, 0.0, -0.0, 1e-45, -1e-45, 3e38, -3e38, 1.0, -1.0, 1e-30, 65504.0, 65520.0, 2.0 ** -24, 0.3],
+                   dtype=np.float32)
+    s = np.linspace(-2, 2, 15).astype(np.float32)
+    t = fb.fewbit_table_from_arrays("tanh", 4, s, lev)
+    special = torch.tensor([0.0, -0.0, inf, -inf, nan, 1e-45, 1e-40, -1e-40, 65504.0, 3e38, -3e38, 1.0], device=DEV)
+    gen = torch.Generator(device=DEV).manual_seed(5)
+    for n, scale in ((5000, 1.0), ((1 << 22) + 77, 1e3), (1 << 20, 1e-3)):
+        x = (torch.randn(n, generator=gen, device=DEV) * 1.5).to(TORCH_DT[dtype])
+        g = (torch.randn(n, generator=gen, device=DEV) * scale).to(TORCH_DT[dtype])
+        for at in (0, 100, 300, 1024, n - 12):
+            g[at:at + special.numel()] = special.to(TORCH_DT[dtype])
+        _, pk = fb.fewbit_fwd(t, x)
+        gi = fb.fewbit_bwd(t, pk, g)
+        codes = torch.bucketize(x.float(), torch.from_numpy(s).to(DEV), right=False)
+        want = (g.float() * torch.from_numpy(lev).to(DEV)[codes]).to(TORCH_DT[dtype])
+        assert torch.equal(torch.isnan(gi), torch.isnan(want)), (dtype, n)
+        number = ~torch.isnan(want)
+        assert torch.equal(gi[number].view(torch.uint8), want[number].view(torch.uint8)), (dtype, n)
+
+
 @pytest.mark.parametrize("seed", [6, 7])
 def test_randomised_folded_tables_under_every_variant(seed, monkeypatch):
     """Folded tables (caption of Fig. 3) with random range and grid, random dtype, size and input
