@@ -651,12 +651,9 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     const unsigned n_long = short_blocks ? static_cast<unsigned>(long_ctas) : grid;
     // Programmatic dependent launch lets this grid's CTAs take their places while the previous kernel
     // of the stream drains (they wait there for it to complete): back-to-back launches of small
-    // tensors go from 4.2 us to ~2 us apiece.  The exception: an issue-bound binary32 activation
-    // whose grid lies between one CTA per SM and a full wave -- there the early CTAs pile up on the
-    // SMs the previous kernel left idle and the grid then runs on part of the SMs (binary32 GELU,
-    // 2^20 elements: 8.3 -> 9.2 us); up to one CTA per SM nothing can pile up.
-    const bool issue_bound = sizeof(T) == 4 && act_weight(ACT) == 2;
-    const bool pdl = pdl_enabled() && (!issue_bound || grid <= static_cast<unsigned>(sms) || grid >= static_cast<unsigned>(slots));
+    // tensors go from 4.2 us to ~2 us apiece, and no size or activation measured slower with it
+    // (batches of 8 launches, 2^16 .. 2^28 elements).
+    const bool pdl = pdl_enabled();
     return launch_pdl(kernel, grid, static_cast<unsigned>(warps_per_cta * 32), smem * warps_per_cta / (kFwdThreads / 32), st, pdl,
                       p2, static_cast<const T *>(x), static_cast<T *>(y), packed, n, static_cast<int>(iters), n_long);
 }
