@@ -7,10 +7,15 @@ workload: for every bit width of the workload, the fused forward kernel
 level lookup + multiply).  Prints ONE JSON line (rank 0).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c3|c2|c4|c1]
+                    [--scaling weak|strong]
 
-N > 1 is launched by torchrun; every rank processes its own tensor of the
-workload's shape (the path is elementwise: independent shards, no collective
-on the data path), time is the max over ranks.
+N > 1: one rank per GPU.  Under torchrun (WORLD_SIZE set) the script is a rank; started plainly with
+--gpus N > 1 it re-launches itself under torch.distributed.run with N ranks on 127.0.0.1.  The path is
+elementwise, so the ranks share nothing but the barrier and the max-reduction of the time: with
+--scaling weak (default) every rank processes its own tensor of the workload's shape, with --scaling
+strong ONE tensor of the workload is cut with workloads.shard_range on multiples of 32 elements and
+every rank runs its shard; `checksum` (a sum over the bit patterns of every output) is then the same
+for every N.
 """
 from __future__ import annotations
 
@@ -137,9 +142,23 @@ def dist_setup(n_gpus: int):
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("NCCL_DEBUG", "INFO")          # the communicator log shows the rank count
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
         torch.cuda.set_device(local)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     return rank, world, local
+
+
+def spawn_ranks(n_gpus: int) -> int:
+    """Started without torchrun but with --gpus N > 1: run this very command line as N ranks of one
+    node (rendezvous on 127.0.0.1, a free port) and return the launcher's exit code."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd)
 
 
 def barrier(world: int):
@@ -236,6 +255,7 @@ def run_reference(args, case: wl.Case, act: str):
     value = passes / t
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "elements/s", "n_gpus": args.gpus,
+        "ranks_started": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": case.dtype, "data": "synthetic",
         "config": {"workload": case.name, "act": act, "bits": list(case.bits), "elements_per_step_sample": sample,
@@ -261,8 +281,20 @@ def run_ours(args, case: wl.Case, act: str):
     torch.cuda.set_device(dev)
     fb.load_library()
 
-    n = args.elements or case.n
-    x, g = wl.draw(dataclass_replace_seed(case, case.seed + rank), dev, n=n)
+    n_total = args.elements or case.n
+    strong = args.scaling == "strong"
+    if strong:
+        # one tensor for the whole job (every rank draws it with the same seed), cut on multiples of
+        # 32 elements: each shard's packed words are whole, no rank touches another's data
+        xf, gf = wl.draw(case, dev, n=n_total)
+        lo, hi = wl.shard_range(n_total, rank, world, align=32)
+        x, g = xf[lo:hi].clone(), gf[lo:hi].clone()
+        del xf, gf
+        torch.cuda.empty_cache()
+        n = hi - lo
+    else:
+        n = n_total
+        x, g = wl.draw(dataclass_replace_seed(case, case.seed + rank), dev, n=n)
     y, gi = torch.empty_like(x), torch.empty_like(g)
     tables = {b: fb.fewbit_table_create(act, b) for b in case.bits}
     packed = {b: torch.empty(fb.fewbit_packed_bytes(n, b) // 4, dtype=torch.int32, device=dev) for b in case.bits}
@@ -335,9 +367,26 @@ def run_ours(args, case: wl.Case, act: str):
                 "frac_of_nominal_8TBs": per_kernel[dom]["gbs"] / NOMINAL_HBM_GBS,
                 "traffic": NCU_TRAFFIC_BYTES_PER_ELEM.get((case.dtype, dom)) and
                 NCU_TRAFFIC_BYTES_PER_ELEM[(case.dtype, dom)] * n}
-    elems_per_step = 2 * len(case.bits) * n
-    value = world * elems_per_step * args.steps / (total_ms * 1e-3)
-    bytes_per_step = 2 * sum(algorithmic_bytes(case, n, b) for b in case.bits)
+    n_job = n_total if strong else world * n                   # elements all ranks process per kernel pass
+    elems_per_step = 2 * len(case.bits) * n_job
+    value = elems_per_step * args.steps / (total_ms * 1e-3)
+    bytes_per_step = 2 * sum(algorithmic_bytes(case, n_job, b) for b in case.bits)
+    # Sum over the bit patterns of every output of one step (y and grad_in of the last bit width, the
+    # packed words of every width), added up over the ranks: with --scaling strong it does not depend on N.
+    xs0, gs0, ys0, gis0, ps0 = bufs[0]
+    iview = torch.int32 if case.dtype == "f32" else torch.int16
+    checksum = 0
+    for b in case.bits:
+        fb.fewbit_fwd(tables[b], xs0, ys0, ps0[b])
+        checksum += int(ps0[b].to(torch.int64).sum().item())
+    fb.fewbit_bwd(tables[case.bits[-1]], ps0[case.bits[-1]], gs0, gis0)
+    checksum += int(ys0.view(iview).to(torch.int64).sum().item()) + int(gis0.view(iview).to(torch.int64).sum().item())
+    if world > 1:
+        import torch.distributed as dist
+        cs = torch.tensor([checksum], dtype=torch.int64, device=dev)
+        dist.all_reduce(cs)
+        checksum = int(cs.item())
+    checksum &= (1 << 63) - 1
 
     # ---- end to end through the host-buffer entry points -----------------------------------------
     e2e = None
@@ -362,7 +411,7 @@ def run_ours(args, case: wl.Case, act: str):
         eb = elem_size(case)
         h2d = sum(n * eb + (n * eb + packed[b].numel() * 4) for b in case.bits)
         d2h = sum((n * eb + packed[b].numel() * 4) + n * eb for b in case.bits)
-        e2e = {"value": world * elems_per_step * args.e2e_steps / secs, "unit": "elements/s",
+        e2e = {"value": elems_per_step * args.e2e_steps / secs, "unit": "elements/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
                "gbs_pcie_each_way": h2d * args.e2e_steps / secs / 1e9,
                "api": "fewbit_fwd_host / fewbit_bwd_host on pinned host tensors"}
@@ -384,6 +433,9 @@ def run_ours(args, case: wl.Case, act: str):
         f16 = dataclasses.replace(wl.C3, name="c3_shape_f16_2p26", dtype="f16", shape=(1 << 26,), bits=(1, 4))
         also["f16"] = quick_config(fb, f16, dev, reps=5)                   # IEEE binary16 storage
         also["c2_bias"] = quick_config(fb, wl.C2, dev, bias_cols=wl.C2.shape[-1])   # f(x + bias), the add inside the kernel
+        del x, g, y, gi, packed, bufs, xs0, gs0, ys0, gis0, ps0
+        torch.cuda.empty_cache()
+        also["c5"] = c5_summary(fb, dev, peak)                              # the sweep at >= 16 M elements, compact
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
@@ -392,17 +444,19 @@ def run_ours(args, case: wl.Case, act: str):
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "elements/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": args.scaling,
             "vs_baseline": None, "dtype": case.dtype, "data": "synthetic",
             "config": {"workload": case.name if not args.elements else f"{case.name} cut to {n} elements",
-                       "act": act, "bits": list(case.bits), "shape": list(case.shape) if not args.elements else [n],
-                       "elements": n, "launches_per_step": len(order),
+                       "act": act, "bits": list(case.bits), "shape": list(case.shape) if not args.elements else [n_total],
+                       "elements": n_job, "elements_per_rank": n, "launches_per_step": len(order),
                        "l2": "inputs larger than L2 (no flush)" if sets == 1 else f"cold by rotation over {sets} copies of the buffers ({sets * footprint / 2 ** 20:.0f} MiB), a different one every launch; launches queued behind a device-side delay",
                        "elements_counted": "once per kernel pass (forward and backward each count n)",
-                       "parallelism": f"independent shards x{world}"},
-            "hbm_gbs": world * bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9,
-            "hbm_frac_of_nominal_8TBs": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-            "hbm_frac_of_measured_copy": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9 / peak,
+                       "parallelism": (f"one tensor cut into {world} shards on multiples of 32 elements" if strong
+                                       else f"independent tensors x{world}") + ", no collective on the data path"},
+            "checksum": checksum,
+            "hbm_gbs": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9,
+            "hbm_frac_of_nominal_8TBs": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS / world,
+            "hbm_frac_of_measured_copy": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9 / peak / world,
             "roofline": roofline, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches_in_region, "clocks": clocks, "torch_unfused": torch_ref, "also": also,
             "saved_activation_ratio": {str(b): 8 * elem_size(case) / b for b in case.bits},
@@ -413,11 +467,10 @@ def run_ours(args, case: wl.Case, act: str):
         dist.destroy_process_group()
 
 
-# DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum of one launch / n) read from the
-# ncu captures summarised under profiles/; None until a capture exists for that kernel.
+# DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum of one launch / n) from the ncu
+# captures of the 2^27-element launches of these kernels; None for a kernel without a capture.
 NCU_TRAFFIC_BYTES_PER_ELEM = {
-    # profiles/fwd_kernel_gelu_k4_bf16_2p27.md and profiles/bwd_kernel_k4_bf16_2p27.md (2^27 elements;
-    # scaled per element: a lower bound for the full launch, the L2 keeps ~55 MB of dirty lines either way)
+    # scaled per element: a lower bound for the full launch, the L2 keeps ~55 MB of dirty lines either way
     ("bf16", "fwd_k4"): 4.097,
     ("bf16", "bwd_k4"): 4.101,
     ("bf16", "fwd_k1"): 3.731,
@@ -524,6 +577,25 @@ def quick_config(fb, case: wl.Case, dev, reps: int = 10, folded: bool = False, b
             "launches_per_timing": inner, "cases": out}
 
 
+def c5_summary(fb, dev, peak: float, sizes=(2 ** 24, 2 ** 24 + 7, 2 ** 28), reps: int = 3):
+    """Config 5 at the sizes of at least 16 M elements, compact: per size and dtype, for every bit
+    width the minimum and the median over the seven activations of the forward and backward fraction
+    of the copy bandwidth (`peak`), the activation with the slowest forward, and what a torch copy_
+    with the traffic of the 2-bit kernels reaches at that size, timed the same way."""
+    out = {}
+    for case in wl.sweep_cases(sizes):
+        r = quick_config(fb, case, dev, reps=reps)["cases"]
+        row = {"copy_same_traffic_frac": round(copy_at_size(int(algorithmic_bytes(case, case.n, 2)) // 2, dev, reps=reps) / peak, 3)}
+        for kind in ("fwd", "bwd"):
+            per_bits = [[r[f"{a}_k{b}"][f"{kind}_gbs"] / peak for a in case.acts] for b in case.bits]
+            row[f"{kind}_frac_min"] = [round(min(v), 3) for v in per_bits]
+            row[f"{kind}_frac_median"] = [round(statistics.median(v), 3) for v in per_bits]
+        row["slowest_fwd"] = [min(case.acts, key=lambda a: r[f"{a}_k{b}"]["fwd_gbs"]) for b in case.bits]
+        out[f"{case.dtype}_{case.n}"] = row
+        torch.cuda.empty_cache()
+    return {"bits": [1, 2, 3, 4], "activations": list(wl.ACTIVATIONS), "frac_of": f"{peak} GB/s", "cases": out}
+
+
 def copy_at_size(nbytes: int, dev, reps: int = 10):
     """GB/s of a torch copy_ that reads nbytes and writes nbytes, timed like quick_config (L2-cold by
     rotation, short launches as a back-to-back batch): what a plain copy reaches at a given size."""
@@ -566,6 +638,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--scaling", choices=["weak", "strong"], default="weak",
+                    help="N > 1: weak = a tensor of the workload per rank; strong = one tensor cut into N shards")
     ap.add_argument("--workload", choices=sorted(wl.CONFIGS), default="c3")
     ap.add_argument("--act", default=None, help="activation of the workload to time (default: its first)")
     ap.add_argument("--elements", type=int, default=0,
@@ -580,6 +654,8 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="time config 5 (7 activations x 1-4 bits x bf16/fp32 at 2^16, 2^20, 2^24, 2^24+7 and 2^28 elements) instead")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
     if args.sweep:
         return run_sweep(args)
     args.warmup = max(args.warmup, 0)

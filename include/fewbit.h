@@ -178,10 +178,15 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  *     y[e]      = f(x[e])                 exact activation, rounded to dtype
  *     code[e]   = #{ j : s[j] < x[e] }    Eq. 2 / the sorted search of Listing 1
  *     packed    = the codes as a `bits`-bit stream (layout above)
- * x, y: DEVICE, n elements of `dtype`, 32-byte aligned; y == x (exact alias)
+ * x, y: DEVICE, n elements of `dtype`, 16-byte aligned; y == x (exact alias)
  * is allowed, any other overlap is undefined.  packed: DEVICE,
- * fewbit_packed_bytes(n, bits) bytes, 16-byte aligned; nothing beyond those
+ * fewbit_packed_bytes(n, bits) bytes, 4-byte aligned; nothing beyond those
  * bytes is written.  n == 0 returns FEWBIT_OK without a launch.
+ * (Alignment beyond the rule only widens the accesses: binary32 buffers that
+ * are all 32-byte aligned move 256 bits per lane instead of 2 x 128, packed
+ * words that are 8-byte (2 bits) or 16-byte (4 bits) aligned are stored as one
+ * vector.  Any view of a tensor that starts on a multiple of 32 elements
+ * therefore satisfies the rule for x, y and packed at once.)
  * Errors: FEWBIT_ERR_INVALID_ARG (NULL table or buffer, bad dtype),
  * FEWBIT_ERR_ALIGNMENT, FEWBIT_ERR_CUDA (launch failed).
  * The interval search has several equivalent kernel variants (binary search,
@@ -194,16 +199,13 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  * first such call on a device creates up to 16 CUDA events, and each call
  * records one after its kernel).  While `stream` is being captured,
  * or when all sets are in use by other streams, the kernel falls back to a
- * static partition: same results, ~10 % slower.  Environment variables for
- * testing and tuning only: FEWBIT_FWD_TABLE = always | never | auto (use of
- * the code-table variant, default auto), FEWBIT_FWD_QUEUE = never (static
- * partition), FEWBIT_FWD_ITERS = <k> (warp-blocks per warp) and
- * FEWBIT_FWD_WARPS = <w> (warps per CTA of the variants without a code table).
+ * static partition: same results, ~10 % slower.  The choices can be overridden
+ * for testing and tuning with fewbit_set_option (below); the library reads no
+ * environment variable.
  * Both device kernels are launched with programmatic stream serialization:
  * their CTAs may be scheduled while the previous kernel of `stream` drains,
  * and wait there for its completion before they touch memory, so stream order
- * holds as usual (FEWBIT_PDL=0 in the environment launches them the ordinary
- * way).
+ * holds as usual (FEWBIT_OPT_PDL = 0 launches them the ordinary way).
  */
 FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y,
                                     uint32_t *packed, size_t n, fewbit_dtype dtype, void *stream);
@@ -218,8 +220,8 @@ FEWBIT_API fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, vo
  * respect to the bias.
  *
  * x, y: DEVICE, rows * cols elements; bias: DEVICE, cols elements of `dtype`,
- * 32-byte aligned like x and y; packed: DEVICE, fewbit_packed_bytes(rows * cols,
- * bits) bytes, 16-byte aligned.  y may alias x exactly.  cols must be a multiple
+ * 16-byte aligned like x and y; packed: DEVICE, fewbit_packed_bytes(rows * cols,
+ * bits) bytes, 4-byte aligned.  y may alias x exactly.  cols must be a multiple
  * of 8 below 2^32 (a lane's 8 consecutive elements then never straddle a row
  * end) and the table must not be a folded one, else FEWBIT_ERR_UNSUPPORTED;
  * rows * cols == 0 is a no-op.  Asynchronous on `stream`, allocates nothing; same kernel
@@ -236,8 +238,8 @@ FEWBIT_API fewbit_status fewbit_fwd_bias(const fewbit_table *table, const void *
  *     grad_in[e] = round_dtype( (float)grad_out[e] * lev[code[e]] )
  * (Eq. 1 with f' replaced by q of Eq. 2; one binary32 multiply, one rounding).
  * packed: DEVICE, as written by fewbit_fwd with a table of the same `bits`,
- * 16-byte aligned.  grad_out, grad_in: DEVICE, n elements of `dtype`,
- * 32-byte aligned; grad_in == grad_out allowed.  Errors as fewbit_fwd.
+ * 4-byte aligned.  grad_out, grad_in: DEVICE, n elements of `dtype`,
+ * 16-byte aligned; grad_in == grad_out allowed.  Errors as fewbit_fwd.
  */
 FEWBIT_API fewbit_status fewbit_bwd(const fewbit_table *table, const uint32_t *packed,
                                     const void *grad_out, void *grad_in, size_t n,
@@ -313,8 +315,48 @@ FEWBIT_API fewbit_status fewbit_fwd_host_static(const fewbit_table *table, const
                                                 fewbit_dtype dtype, void *stream);
 
 /* ------------------------------------------------------------------------- */
-/* Diagnostics                                                                */
+/* Options and diagnostics                                                    */
 /* ------------------------------------------------------------------------- */
+
+/*
+ * Process-wide switches for testing and tuning (the paper has no counterpart;
+ * every setting gives the same results, only the kernel variant or the launch
+ * geometry changes).  Stored in atomics: may be set from any thread at any
+ * time and apply to the launches that follow.
+ *   FEWBIT_OPT_FWD_TABLE    0 size-based choice (default), 1 the shared-memory
+ *                           code-table variant whenever the table has one,
+ *                           2 never;
+ *   FEWBIT_OPT_FWD_QUEUE    0 lease work counters when possible (default),
+ *                           1 always the static partition;
+ *   FEWBIT_OPT_FWD_ITERS    0 size-based (default), 1..64 warp-blocks per warp;
+ *   FEWBIT_OPT_FWD_WARPS    0 default, 1..16 warps per CTA of the variants
+ *                           without a code table (values beyond what the kernel
+ *                           is compiled for are ignored);
+ *   FEWBIT_OPT_PDL          1 programmatic dependent launch (default), 0 off;
+ *   FEWBIT_OPT_COUNT_TAILS  1: every warp that runs the forward kernel's
+ *                           ragged-tail path adds one to a device counter read
+ *                           by fewbit_tail_warp_count (default 0: no counting).
+ * fewbit_set_option returns FEWBIT_ERR_INVALID_ARG for an unknown option or a
+ * value outside its range; fewbit_get_option returns -1 for an unknown option.
+ */
+typedef enum fewbit_option {
+    FEWBIT_OPT_FWD_TABLE = 0,
+    FEWBIT_OPT_FWD_QUEUE = 1,
+    FEWBIT_OPT_FWD_ITERS = 2,
+    FEWBIT_OPT_FWD_WARPS = 3,
+    FEWBIT_OPT_PDL = 4,
+    FEWBIT_OPT_COUNT_TAILS = 5
+} fewbit_option;
+FEWBIT_API fewbit_status fewbit_set_option(fewbit_option option, int value);
+FEWBIT_API int fewbit_get_option(fewbit_option option);
+
+/*
+ * Diagnostic: *count (HOST) receives how many warps have run the ragged-tail
+ * path of the forward kernel on the current device while FEWBIT_OPT_COUNT_TAILS
+ * was 1 (exactly one per launch whose n is not a multiple of 1024); reset != 0
+ * clears the counter afterwards.  Synchronises the device.
+ */
+FEWBIT_API fewbit_status fewbit_tail_warp_count(uint64_t *count, int reset);
 
 /* Static, never NULL. */
 FEWBIT_API const char *fewbit_status_string(fewbit_status status);

@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     fewbit_packed_bytes, fewbit_fwd, fewbit_fwd_bias, fewbit_bwd, fewbit_fwd_host, fewbit_bwd_host,
     fewbit_host_workspace_bytes, fewbit_launch_count, library_path, load_library,
     fewbit_fwd_host_static, fewbit_static_max_elements, fewbit_f32_activation_scan,
+    fewbit_set_option, fewbit_get_option, fewbit_tail_warp_count,
 )
 from . import workloads  # noqa: F401
 from .autograd import FewBitActivation, fewbit_activation  # noqa: F401

@@ -84,6 +84,12 @@ def load_library():
     lib.fewbit_last_cuda_error.argtypes = []
     lib.fewbit_launch_count.restype = ctypes.c_uint64
     lib.fewbit_launch_count.argtypes = []
+    lib.fewbit_set_option.restype = ci
+    lib.fewbit_set_option.argtypes = [ci, ci]
+    lib.fewbit_get_option.restype = ci
+    lib.fewbit_get_option.argtypes = [ci]
+    lib.fewbit_tail_warp_count.restype = ci
+    lib.fewbit_tail_warp_count.argtypes = [ctypes.POINTER(ctypes.c_uint64), ci]
     lib.fewbit_f32_activation_scan.restype = ci
     lib.fewbit_f32_activation_scan.argtypes = [ci, ctypes.c_uint64, ctypes.c_uint64, vp, vp]
     _lib = lib
@@ -190,6 +196,33 @@ def fewbit_packed_bytes(n: int, bits: int) -> int:
 
 def fewbit_launch_count() -> int:
     return int(load_library().fewbit_launch_count())
+
+
+OPTIONS = {"fwd_table": 0, "fwd_queue": 1, "fwd_iters": 2, "fwd_warps": 3, "pdl": 4, "count_tails": 5}
+_OPTION_VALUES = {"auto": 0, "always": 1, "never": 2}
+
+
+def fewbit_set_option(option, value) -> None:
+    """Process-wide testing / tuning switch; `option` by name or number, `value` an int (for
+    "fwd_table" also "auto" | "always" | "never"; for "fwd_queue" "auto" | "never")."""
+    opt = OPTIONS[option] if isinstance(option, str) else int(option)
+    if isinstance(value, str):
+        value = {"auto": 0, "never": 1}[value] if opt == 1 else _OPTION_VALUES[value]
+    _check(load_library().fewbit_set_option(opt, int(value)), "fewbit_set_option")
+
+
+def fewbit_get_option(option) -> int:
+    return int(load_library().fewbit_get_option(OPTIONS[option] if isinstance(option, str) else int(option)))
+
+
+def fewbit_tail_warp_count(device=None, reset: bool = False) -> int:
+    """Warps that ran the forward kernel's ragged-tail path on `device` while the "count_tails"
+    option was on.  Synchronises the device."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    out = ctypes.c_uint64()
+    with torch.cuda.device(device):
+        _check(load_library().fewbit_tail_warp_count(ctypes.byref(out), int(reset)), "fewbit_tail_warp_count")
+    return int(out.value)
 
 
 def fewbit_f32_activation_scan(act, first_pattern: int = 0, count: int = 1 << 32, device=None,

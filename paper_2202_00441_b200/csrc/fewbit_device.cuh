@@ -63,13 +63,23 @@ inline cudaError_t launch_pdl(void (*kernel)(Params...), unsigned grid, unsigned
 // ---------------------------------------------------------------------------
 // global memory access: 8 elements per lane, widened to binary32
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void load8(const float *p, float (&v)[8]) {
-    asm volatile("ld.global.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
-                 : "l"(p) : "memory");
+// `wide` (warp-uniform): the address is 32-byte aligned, so the lane-chunk of eight binary32 values
+// moves as one 256-bit access; otherwise (16-byte alignment only) as two 128-bit ones.  The 16-bit
+// types always move 128 bits and ignore the flag.
+__device__ __forceinline__ void load8(const float *p, float (&v)[8], bool wide = true) {
+    if (wide) {
+        asm volatile("ld.global.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                     : "l"(p) : "memory");
+    } else {
+        asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]) : "l"(p) : "memory");
+        asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4+16];"
+                     : "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(p) : "memory");
+    }
 }
 
-__device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&v)[8]) {
+__device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&v)[8], bool = true) {
     uint32_t r[4];
     asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "l"(p) : "memory");
@@ -80,10 +90,15 @@ __device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&v)[8]) {
     }
 }
 
-__device__ __forceinline__ void store8(float *p, const float (&v)[8]) {
-    asm volatile("st.global.v8.f32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
-                 :: "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "l"(p)
-                 : "memory");
+__device__ __forceinline__ void store8(float *p, const float (&v)[8], bool wide = true) {
+    if (wide) {
+        asm volatile("st.global.v8.f32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+                     :: "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "l"(p)
+                     : "memory");
+    } else {
+        asm volatile("st.global.v4.f32 [%4], {%0,%1,%2,%3};" :: "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "l"(p) : "memory");
+        asm volatile("st.global.v4.f32 [%4+16], {%0,%1,%2,%3};" :: "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "l"(p) : "memory");
+    }
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -92,13 +107,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return d;
 }
 
-__device__ __forceinline__ void store8(__nv_bfloat16 *p, const float (&v)[8]) {
+__device__ __forceinline__ void store8(__nv_bfloat16 *p, const float (&v)[8], bool = true) {
     const uint32_t a = pack_bf16x2(v[0], v[1]), b = pack_bf16x2(v[2], v[3]);
     const uint32_t c = pack_bf16x2(v[4], v[5]), d = pack_bf16x2(v[6], v[7]);
     asm volatile("st.global.v4.u32 [%4], {%0,%1,%2,%3};" :: "r"(a), "r"(b), "r"(c), "r"(d), "l"(p) : "memory");
 }
 
-__device__ __forceinline__ void load8(const __half *p, float (&v)[8]) {
+__device__ __forceinline__ void load8(const __half *p, float (&v)[8], bool = true) {
     uint32_t r[4];
     asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "l"(p) : "memory");
@@ -116,7 +131,7 @@ __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
     return d;
 }
 
-__device__ __forceinline__ void store8(__half *p, const float (&v)[8]) {
+__device__ __forceinline__ void store8(__half *p, const float (&v)[8], bool = true) {
     const uint32_t a = pack_f16x2(v[0], v[1]), b = pack_f16x2(v[2], v[3]);
     const uint32_t c = pack_f16x2(v[4], v[5]), d = pack_f16x2(v[6], v[7]);
     asm volatile("st.global.v4.u32 [%4], {%0,%1,%2,%3};" :: "r"(a), "r"(b), "r"(c), "r"(d), "l"(p) : "memory");
@@ -216,34 +231,56 @@ __device__ __forceinline__ void words_to_groups(const uint32_t (&w)[BITS], uint3
     }
 }
 
+// `vec` (warp-uniform): the packed buffer is aligned for the vector access of this bit width (8 bytes
+// at 2 bits, 16 at 4); otherwise (4-byte alignment only) the words move one by one.
 template <int BITS>
-__device__ __forceinline__ void store_words(uint32_t *p, const uint32_t (&w)[BITS]) {
+__device__ __forceinline__ void store_words(uint32_t *p, const uint32_t (&w)[BITS], bool vec = true) {
     if constexpr (BITS == 1) {
         asm volatile("st.global.u32 [%0], %1;" :: "l"(p), "r"(w[0]) : "memory");
     } else if constexpr (BITS == 2) {
-        asm volatile("st.global.v2.u32 [%0], {%1,%2};" :: "l"(p), "r"(w[0]), "r"(w[1]) : "memory");
+        if (vec) {
+            asm volatile("st.global.v2.u32 [%0], {%1,%2};" :: "l"(p), "r"(w[0]), "r"(w[1]) : "memory");
+        } else {
+            asm volatile("st.global.u32 [%0], %1;" :: "l"(p), "r"(w[0]) : "memory");
+            asm volatile("st.global.u32 [%0+4], %1;" :: "l"(p), "r"(w[1]) : "memory");
+        }
     } else if constexpr (BITS == 3) {
         asm volatile("st.global.u32 [%0], %1;" :: "l"(p), "r"(w[0]) : "memory");
         asm volatile("st.global.u32 [%0+4], %1;" :: "l"(p), "r"(w[1]) : "memory");
         asm volatile("st.global.u32 [%0+8], %1;" :: "l"(p), "r"(w[2]) : "memory");
-    } else {
+    } else if (vec) {
         asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+    } else {
+        asm volatile("st.global.u32 [%0], %1;" :: "l"(p), "r"(w[0]) : "memory");
+        asm volatile("st.global.u32 [%0+4], %1;" :: "l"(p), "r"(w[1]) : "memory");
+        asm volatile("st.global.u32 [%0+8], %1;" :: "l"(p), "r"(w[2]) : "memory");
+        asm volatile("st.global.u32 [%0+12], %1;" :: "l"(p), "r"(w[3]) : "memory");
     }
 }
 
 template <int BITS>
-__device__ __forceinline__ void load_words(const uint32_t *p, uint32_t (&w)[BITS]) {
+__device__ __forceinline__ void load_words(const uint32_t *p, uint32_t (&w)[BITS], bool vec = true) {
     if constexpr (BITS == 1) {
         asm volatile("ld.global.L1::no_allocate.u32 %0, [%1];" : "=r"(w[0]) : "l"(p) : "memory");
     } else if constexpr (BITS == 2) {
-        asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "l"(p) : "memory");
+        if (vec) {
+            asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "l"(p) : "memory");
+        } else {
+            asm volatile("ld.global.L1::no_allocate.u32 %0, [%1];" : "=r"(w[0]) : "l"(p) : "memory");
+            asm volatile("ld.global.L1::no_allocate.u32 %0, [%1+4];" : "=r"(w[1]) : "l"(p) : "memory");
+        }
     } else if constexpr (BITS == 3) {
         asm volatile("ld.global.L1::no_allocate.u32 %0, [%1];" : "=r"(w[0]) : "l"(p) : "memory");
         asm volatile("ld.global.L1::no_allocate.u32 %0, [%1+4];" : "=r"(w[1]) : "l"(p) : "memory");
         asm volatile("ld.global.L1::no_allocate.u32 %0, [%1+8];" : "=r"(w[2]) : "l"(p) : "memory");
-    } else {
+    } else if (vec) {
         asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "l"(p) : "memory");
+    } else {
+        asm volatile("ld.global.L1::no_allocate.u32 %0, [%1];" : "=r"(w[0]) : "l"(p) : "memory");
+        asm volatile("ld.global.L1::no_allocate.u32 %0, [%1+4];" : "=r"(w[1]) : "l"(p) : "memory");
+        asm volatile("ld.global.L1::no_allocate.u32 %0, [%1+8];" : "=r"(w[2]) : "l"(p) : "memory");
+        asm volatile("ld.global.L1::no_allocate.u32 %0, [%1+12];" : "=r"(w[3]) : "l"(p) : "memory");
     }
 }
 

@@ -64,12 +64,12 @@ template <> struct Raw<float> { float v[8]; };
 template <> struct Raw<__nv_bfloat16> { uint32_t v[4]; };
 template <> struct Raw<__half> { uint32_t v[4]; };
 
-__device__ __forceinline__ void load_raw(const float *p, Raw<float> &r) { load8(p, r.v); }
-__device__ __forceinline__ void load_raw(const __nv_bfloat16 *p, Raw<__nv_bfloat16> &r) {
+__device__ __forceinline__ void load_raw(const float *p, Raw<float> &r, bool wide) { load8(p, r.v, wide); }
+__device__ __forceinline__ void load_raw(const __nv_bfloat16 *p, Raw<__nv_bfloat16> &r, bool) {
     asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]) : "l"(p) : "memory");
 }
-__device__ __forceinline__ void load_raw(const __half *p, Raw<__half> &r) {
+__device__ __forceinline__ void load_raw(const __half *p, Raw<__half> &r, bool) {
     asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]) : "l"(p) : "memory");
 }
@@ -102,20 +102,25 @@ template <typename T> __device__ __forceinline__ float round_to(float v) {     /
     else if constexpr (std::is_same<T, __half>::value) return __half2float(__float2half_rn(v));
     else return v;
 }
-__device__ __forceinline__ void add_bias(Raw<float> &r, const float *b) {
+__device__ __forceinline__ void add_bias(Raw<float> &r, const float *b, bool wide) {
     float v[8];
-    asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(b));
+    if (wide) {
+        asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(b));
+    } else {
+        asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]) : "l"(b));
+        asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4+16];" : "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(b));
+    }
 #pragma unroll
     for (int e = 0; e < 8; ++e) r.v[e] = __fadd_rn(r.v[e], v[e]);
 }
-__device__ __forceinline__ void add_bias(Raw<__nv_bfloat16> &r, const __nv_bfloat16 *b) {
+__device__ __forceinline__ void add_bias(Raw<__nv_bfloat16> &r, const __nv_bfloat16 *b, bool) {
     uint32_t v[4];
     asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "l"(b));
 #pragma unroll
     for (int i = 0; i < 4; ++i) asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r.v[i]) : "r"(r.v[i]), "r"(v[i]));   // one rounding per half
 }
-__device__ __forceinline__ void add_bias(Raw<__half> &r, const __half *b) {
+__device__ __forceinline__ void add_bias(Raw<__half> &r, const __half *b, bool) {
     uint32_t v[4];
     asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "l"(b));
 #pragma unroll
@@ -223,7 +228,11 @@ struct FwdParams {
     uint32_t cols;                   // with a bias: the row length, a multiple of kLaneElems (a lane-chunk never straddles a row end)
     uint64_t chunks_magic;           // floor(2^64 / (cols / kLaneElems)) + 1: exact division of 32-bit chunk numbers by a multiply-high
     uint32_t long_iters;             // warp-blocks per warp of the long CTAs of a static partition
+    uint32_t flags;                  // kWideData | kVecPacked: what the alignment of the caller's buffers allows
+    unsigned int *tail_counter;      // diagnostic (FEWBIT_OPT_COUNT_TAILS): counts the warps that run the ragged-tail path, or NULL
 };
+constexpr uint32_t kWideData = 1;    // x, y (and bias) are 32-byte aligned: binary32 lane-chunks move as one 256-bit access
+constexpr uint32_t kVecPacked = 2;   // packed is aligned for the vector store of this bit width (8 bytes at 2 bits, 16 at 4)
 
 // ---------------------------------------------------------------------------
 // packed search: codes of the two bfloat16 elements of `x2`, low element in
@@ -288,6 +297,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     const float *thr = reinterpret_cast<const FwdSmem *>(smem_raw + kCells)->thr;
 
     const int lane = threadIdx.x & 31;
+    const bool wide = prm.flags & kWideData, vec = prm.flags & kVecPacked;
     const size_t warps = blockDim.x >> 5;                                        // stride between a warp's warp-blocks (<= kFwdThreads / 32)
     // Static partition: the first long_ctas CTAs own warps * iters warp-blocks each, the rest of the
     // grid warps * 1 (short CTAs at the end of the launch order fill the tail that the long ones
@@ -348,8 +358,8 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     [[maybe_unused]] uint32_t pair_table = 0;
     if constexpr (kIsBf16 && !LUT && BITS == 4) {
         __shared__ uint32_t last_pair[64];
-        if (threadIdx.x < 64)
-            last_pair[threadIdx.x] = (prm.sb2[2 * (threadIdx.x >> 3)] & 0x0000ffffu) | (prm.sb2[2 * (threadIdx.x & 7)] & 0xffff0000u);
+        for (uint32_t i = threadIdx.x; i < 64; i += blockDim.x)           // a CTA may be a single warp
+            last_pair[i] = (prm.sb2[2 * (i >> 3)] & 0x0000ffffu) | (prm.sb2[2 * (i & 7)] & 0xffff0000u);
         __syncthreads();
         pair_table = static_cast<uint32_t>(__cvta_generic_to_shared(last_pair));
     }
@@ -374,7 +384,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     } else if (wb < full) {
         const T *px = x + wb * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
 #pragma unroll
-        for (int t = 0; t < kTilesPerWarp; ++t) load_raw(px + t * kTileElems, cur[t]);
+        for (int t = 0; t < kTilesPerWarp; ++t) load_raw(px + t * kTileElems, cur[t], wide);
     }
     if constexpr (LUT && !kExpandFirst) {                           // expanded while the first loads are in flight
         FwdSmem &sm = *reinterpret_cast<FwdSmem *>(smem_raw + kCells);
@@ -406,11 +416,11 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
             if constexpr (kStages > 0) load_raw_shared(ring + stage * kStageBytes + t * (32 * kChunkBytes), cur[t]);
             if constexpr (BIAS) {
                 if (one_row) {
-                    add_bias(cur[t], static_cast<const T *>(prm.bias) + col0 + t * kTileElems);
+                    add_bias(cur[t], static_cast<const T *>(prm.bias) + col0 + t * kTileElems, wide);
                 } else {
                     uint64_t col = col0 + static_cast<uint64_t>(t) * kTileElems;
                     if (col >= prm.cols) col = prm.cols >= kWarpElems ? col - prm.cols : col % prm.cols;
-                    add_bias(cur[t], static_cast<const T *>(prm.bias) + col);
+                    add_bias(cur[t], static_cast<const T *>(prm.bias) + col, wide);
                 }
             }
             float o[8];
@@ -461,9 +471,9 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
                 }
             }
             grp[t] = g;
-            store8(py + t * kTileElems, o);
+            store8(py + t * kTileElems, o, wide);
             if constexpr (kStages == 0) {
-                if (more) load_raw(px_next + t * kTileElems, cur[t]);
+                if (more) load_raw(px_next + t * kTileElems, cur[t], wide);
             }
         }
         if constexpr (kStages > 0) {                               // refill the stage just consumed
@@ -480,16 +490,18 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         quad_transpose(grp, lane);
         uint32_t w[BITS];
         groups_to_words<BITS>(grp, w);
-        store_words<BITS>(packed + wb * (32 * BITS) + (lane & 3) * (8 * BITS) + (lane >> 2) * BITS, w);
+        store_words<BITS>(packed + wb * (32 * BITS) + (lane & 3) * (8 * BITS) + (lane >> 2) * BITS, w, vec);
         wb = nxt;
         nxt = nxt2;
     }
 
-    // ragged tail: the warp whose sequence reaches the index of the last, partial warp-block; a lane
-    // owns 32 consecutive elements = BITS words
+    // ragged tail: the one warp whose sequence warp0, warp0 + warps, ... reaches the index of the last,
+    // partial warp-block (all_full >= warp0 keeps the unsigned difference from wrapping: 2^64 is not a
+    // multiple of every CTA width); a lane owns 32 consecutive elements = BITS words
     const bool owns_tail = dynamic ? (blockIdx.x == 0 && threadIdx.x < 32)
-                                   : (all_full >= cta_begin && all_full < cta_end && (all_full - warp0) % warps == 0);
+                                   : (all_full >= warp0 && all_full < cta_end && (all_full - warp0) % warps == 0);
     if ((n % kWarpElems) != 0 && owns_tail) {
+        if (prm.tail_counter != nullptr && lane == 0) atomicAdd(prm.tail_counter, 1u);
         const size_t full = all_full;
         const size_t base = full * kWarpElems + static_cast<size_t>(lane) * 32;
         uint32_t w[BITS + 1];
@@ -564,9 +576,9 @@ constexpr int act_weight(int act) {
          : (act == FEWBIT_GELU || act == FEWBIT_SILU) ? 2 : 1;
 }
 constexpr size_t kLutMinIters = 8;      // below this many warp-blocks per warp the table does not pay for its expansion
-const char *fwd_iters_override();        // tuning aid: environment FEWBIT_FWD_ITERS
-bool pdl_enabled();
-const char *fwd_warps_override();        // tuning aid: environment FEWBIT_FWD_WARPS (variant without a table)
+int fwd_iters_override();                // FEWBIT_OPT_FWD_ITERS: 0 = the size-based choice
+bool pdl_enabled();                      // FEWBIT_OPT_PDL
+int fwd_warps_override();                // FEWBIT_OPT_FWD_WARPS (variants without a table): 0 = the default
 
 template <int ACT, int BITS, typename T, bool LUT, bool FOLD, bool BIAS = false>
 cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *packed, size_t n, cudaStream_t st) {
@@ -594,10 +606,8 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     size_t warps_per_cta = kFwdThreads / 32;
     if constexpr (!LUT) {
         warps_per_cta = 4;
-        if (const char *w = fwd_warps_override()) {
-            const int v = atoi(w);
-            if (v >= 1 && v <= kFwdThreads / 32) warps_per_cta = static_cast<size_t>(v);
-        }
+        const int v = fwd_warps_override();
+        if (v >= 1 && v <= kFwdThreads / 32) warps_per_cta = static_cast<size_t>(v);
     }
     const size_t warp_blocks = n / kWarpElems + ((n % kWarpElems) ? 1 : 0);
     // Iterations per warp.  Without a table: two from about 1.5 waves of resident warps on (the
@@ -631,7 +641,7 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
         iters = sizeof(T) == 2 ? warp_blocks * 2 / (warps_per_cta * slots * 3) : 1;
         iters = iters < 1 ? 1 : (iters > 4 ? 4 : iters);
     }
-    if (const char *dbg = fwd_iters_override()) iters = static_cast<size_t>(atoi(dbg));
+    if (const int forced = fwd_iters_override(); forced >= 1) iters = static_cast<size_t>(forced);
     // When the CTAs take several warp-blocks per warp, the last wave's worth of warp-blocks goes to
     // short CTAs (one warp-block per warp) at the end of the launch order: they fill the tail that
     // the long CTAs leave when they finish at different times (2^26 elements: 50.2 -> 48.1 us,

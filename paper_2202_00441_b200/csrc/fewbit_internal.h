@@ -67,6 +67,10 @@ cudaError_t queue_acquire(cudaStream_t stream, QueueLease *lease);
 // After the kernel launch (also after a failed one): records the point of `stream` up to which
 // the set is in use.
 cudaError_t queue_release(const QueueLease &lease, cudaStream_t stream);
+// Diagnostic counter of the warps that ran the forward kernel's ragged-tail path (one word of the
+// same file-scope device array): its device address on the current device, and a synchronising read.
+cudaError_t tail_counter_address(unsigned int **out);
+cudaError_t tail_counter_read(uint64_t *count, bool reset);
 }  // namespace fewbit
 
 // The parameters s and y of Eq. 2, as binary32.  Unused boundary slots hold

@@ -14,23 +14,24 @@ thread_local int t_last_cuda_error = 0;
 // ---------------------------------------------------------------------------
 template <int BITS, typename T>
 __global__ void __launch_bounds__(kThreads)
-bwd_kernel(const __grid_constant__ Levels tl, const uint32_t *packed, const T *grad_out, T *grad_in, size_t n) {
+bwd_kernel(const __grid_constant__ Levels tl, const uint32_t *packed, const T *grad_out, T *grad_in, size_t n, uint32_t flags) {
     pdl_launch_dependents();
     __shared__ float lev[kMaxLevels];
     if (threadIdx.x < kMaxLevels) lev[threadIdx.x] = tl.lev[threadIdx.x];
     __syncthreads();
     pdl_wait();
     const int lane = threadIdx.x & 31;
+    const bool wide = flags & kWideData, vec = flags & kVecPacked;
     const size_t wb = static_cast<size_t>(blockIdx.x) * kWarpsPerCta + (threadIdx.x >> 5);
     const size_t full = n / kWarpElems;
     constexpr uint32_t kMask = (1u << BITS) - 1u;
     if (wb < full) {
         const size_t base = wb * kWarpElems + static_cast<size_t>(lane) * kLaneElems;
         uint32_t w[BITS];
-        load_words<BITS>(packed + wb * (32 * BITS) + (lane & 3) * (8 * BITS) + (lane >> 2) * BITS, w);
+        load_words<BITS>(packed + wb * (32 * BITS) + (lane & 3) * (8 * BITS) + (lane >> 2) * BITS, w, vec);
         float v[kTilesPerWarp][8];
 #pragma unroll
-        for (int t = 0; t < kTilesPerWarp; ++t) load8(grad_out + base + t * kTileElems, v[t]);
+        for (int t = 0; t < kTilesPerWarp; ++t) load8(grad_out + base + t * kTileElems, v[t], wide);
         uint32_t grp[4];
         words_to_groups<BITS>(w, grp);
         quad_transpose(grp, lane);
@@ -39,7 +40,7 @@ bwd_kernel(const __grid_constant__ Levels tl, const uint32_t *packed, const T *g
             float o[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) o[e] = __fmul_rn(v[t][e], lev[(grp[t] >> (BITS * e)) & kMask]);
-            store8(grad_in + base + t * kTileElems, o);
+            store8(grad_in + base + t * kTileElems, o, wide);
         }
     } else if (wb == full && (n % kWarpElems) != 0) {
         const size_t base = full * kWarpElems + static_cast<size_t>(lane) * 32;
@@ -64,7 +65,7 @@ bwd_kernel(const __grid_constant__ Levels tl, const uint32_t *packed, const T *g
 // ---------------------------------------------------------------------------
 // dispatch
 // ---------------------------------------------------------------------------
-using BwdLaunch = cudaError_t (*)(const Levels &, const uint32_t *, const void *, void *, size_t, cudaStream_t);
+using BwdLaunch = cudaError_t (*)(const Levels &, const uint32_t *, const void *, void *, size_t, uint32_t, cudaStream_t);
 
 inline unsigned bwd_grid_for(size_t n) {
     const size_t warps = n / kWarpElems + ((n % kWarpElems) ? 1 : 0);
@@ -72,8 +73,8 @@ inline unsigned bwd_grid_for(size_t n) {
 }
 
 template <int BITS, typename T>
-cudaError_t launch_bwd(const Levels &tl, const uint32_t *packed, const void *g, void *gi, size_t n, cudaStream_t st) {
-    return launch_pdl(bwd_kernel<BITS, T>, bwd_grid_for(n), kThreads, 0, st, pdl_enabled(), tl, packed, static_cast<const T *>(g), static_cast<T *>(gi), n);
+cudaError_t launch_bwd(const Levels &tl, const uint32_t *packed, const void *g, void *gi, size_t n, uint32_t flags, cudaStream_t st) {
+    return launch_pdl(bwd_kernel<BITS, T>, bwd_grid_for(n), kThreads, 0, st, pdl_enabled(), tl, packed, static_cast<const T *>(g), static_cast<T *>(gi), n, flags);
 }
 
 const BwdLaunch kBwd[kMaxBits][3] = {      // [bits - 1][dtype: f32, bf16, f16]
@@ -125,22 +126,27 @@ int device_sm_count(cudaError_t *err) {
     return sms;
 }
 
-const char *fwd_iters_override() {
-    static const char *v = getenv("FEWBIT_FWD_ITERS");
-    return (v && *v) ? v : nullptr;
-}
+// Process-wide options (fewbit_set_option): plain atomics, read with relaxed loads on every launch.
+// No environment variable is read anywhere in the library.
+constexpr int kNumOptions = 6;
+std::atomic<int> g_option[kNumOptions] = {{0}, {0}, {0}, {0}, {1}, {0}};   // defaults; FEWBIT_OPT_PDL is on
+inline int option(fewbit_option o) { return g_option[o].load(std::memory_order_relaxed); }
 
-bool pdl_enabled() {
-    static const bool on = [] { const char *v = getenv("FEWBIT_PDL"); return !(v && v[0] == '0'); }();   // testing aid: FEWBIT_PDL=0
-    return on;
-}
-
-const char *fwd_warps_override() {
-    static const char *v = getenv("FEWBIT_FWD_WARPS");
-    return (v && *v) ? v : nullptr;
-}
+int fwd_iters_override() { return option(FEWBIT_OPT_FWD_ITERS); }
+bool pdl_enabled() { return option(FEWBIT_OPT_PDL) != 0; }
+int fwd_warps_override() { return option(FEWBIT_OPT_FWD_WARPS); }
 
 inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// What the alignment of the caller's buffers allows (the rule itself -- 16 bytes for element
+// buffers, 4 for the packed words -- is checked by the entry points).  a, b, c: the element buffers
+// of the call (c may be NULL).
+inline uint32_t access_flags(const void *a, const void *b, const void *c, const void *packed, int bits) {
+    uint32_t f = 0;
+    if (aligned(a, 32) && aligned(b, 32) && (c == nullptr || aligned(c, 32))) f |= kWideData;
+    if (aligned(packed, bits == 2 ? 8 : 16)) f |= kVecPacked;
+    return f;
+}
 
 }  // namespace fewbit
 
@@ -162,6 +168,12 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
     }
     prm.runs = dtype == FEWBIT_F16 ? table->runs_f16 : (bf16 ? table->runs_bf16 : table->runs_f32);
     prm.queue = nullptr;
+    prm.flags = access_flags(x, y, bias, packed, table->bits);
+    prm.tail_counter = nullptr;
+    if (option(FEWBIT_OPT_COUNT_TAILS) != 0) {
+        const cudaError_t terr = tail_counter_address(&prm.tail_counter);
+        if (terr != cudaSuccess) { t_last_cuda_error = static_cast<int>(terr); return FEWBIT_ERR_CUDA; }
+    }
     // the shared-memory code table pays off only when every warp of a one-wave grid gets enough work
     cudaError_t sm_err = cudaSuccess;
     const size_t slots = static_cast<size_t>(device_sm_count(&sm_err)) * (bf16 ? FwdCtas<__nv_bfloat16, true>::value : FwdCtas<float, true>::value);
@@ -193,10 +205,8 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
         use_lut = (table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && weight >= 1 && waves >= min_waves3);
     }
     bool forced_table = false;
-    if (const char *force = getenv("FEWBIT_FWD_TABLE")) {               // testing aid, see fewbit.h
-        if (force[0] == 'a' && force[1] == 'l') { use_lut = prm.runs.count != 0; forced_table = true; }   // "always"
-        else if (force[0] == 'n') use_lut = false;                        // "never"; anything else ("auto"): the size-based choice
-    }
+    if (const int force = option(FEWBIT_OPT_FWD_TABLE); force == 1) { use_lut = prm.runs.count != 0; forced_table = true; }
+    else if (force == 2) use_lut = false;
     // The table variants distribute their warp-blocks dynamically when a set of work counters can
     // be leased (not during stream capture); the 16-bit types at 3 bits only beat the packed search
     // that way.  binary32 ReLU / leaky ReLU measured faster with short CTAs and a static partition,
@@ -209,8 +219,7 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
     if (launcher(use_lut) == nullptr || launcher(false) == nullptr) return FEWBIT_ERR_UNSUPPORTED;   // before any lease is taken
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     QueueLease lease;
-    const char *queue_mode = getenv("FEWBIT_FWD_QUEUE");               // testing aid: "never" keeps the static partition
-    if (use_lut && (bf16 || (act_weight(table->act) >= 1 && waves >= 2)) && !(queue_mode && queue_mode[0] == 'n')) {
+    if (use_lut && (bf16 || (act_weight(table->act) >= 1 && waves >= 2)) && option(FEWBIT_OPT_FWD_QUEUE) == 0) {
         const cudaError_t qerr = queue_acquire(st, &lease);
         if (qerr != cudaSuccess) { t_last_cuda_error = static_cast<int>(qerr); return FEWBIT_ERR_CUDA; }
         prm.queue = lease.counters;
@@ -237,7 +246,7 @@ fewbit_status fewbit_fwd(const fewbit_table *table, const void *x, void *y, uint
     if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
     if (n == 0) return FEWBIT_OK;
     if (x == nullptr || y == nullptr || packed == nullptr) return FEWBIT_ERR_INVALID_ARG;
-    if (!aligned(x, 32) || !aligned(y, 32) || !aligned(packed, 16)) return FEWBIT_ERR_ALIGNMENT;
+    if (!aligned(x, 16) || !aligned(y, 16) || !aligned(packed, 4)) return FEWBIT_ERR_ALIGNMENT;
     return forward(table, x, nullptr, 0, y, packed, n, dtype, stream);
 }
 
@@ -249,7 +258,7 @@ fewbit_status fewbit_fwd_bias(const fewbit_table *table, const void *x, const vo
     if (x == nullptr || bias == nullptr || y == nullptr || packed == nullptr) return FEWBIT_ERR_INVALID_ARG;
     if (cols % kLaneElems != 0 || cols > 0xffffffffull || table->folded) return FEWBIT_ERR_UNSUPPORTED;
     if (rows > SIZE_MAX / cols) return FEWBIT_ERR_INVALID_ARG;
-    if (!aligned(x, 32) || !aligned(bias, 32) || !aligned(y, 32) || !aligned(packed, 16)) return FEWBIT_ERR_ALIGNMENT;
+    if (!aligned(x, 16) || !aligned(bias, 16) || !aligned(y, 16) || !aligned(packed, 4)) return FEWBIT_ERR_ALIGNMENT;
     return forward(table, x, bias, static_cast<uint32_t>(cols), y, packed, rows * cols, dtype, stream);
 }
 
@@ -259,13 +268,42 @@ fewbit_status fewbit_bwd(const fewbit_table *table, const uint32_t *packed, cons
     if (table == nullptr || !valid_dtype(dtype)) return FEWBIT_ERR_INVALID_ARG;
     if (n == 0) return FEWBIT_OK;
     if (packed == nullptr || grad_out == nullptr || grad_in == nullptr) return FEWBIT_ERR_INVALID_ARG;
-    if (!aligned(grad_out, 32) || !aligned(grad_in, 32) || !aligned(packed, 16)) return FEWBIT_ERR_ALIGNMENT;
+    if (!aligned(grad_out, 16) || !aligned(grad_in, 16) || !aligned(packed, 4)) return FEWBIT_ERR_ALIGNMENT;
     Levels tl;
     for (int m = 0; m < kMaxLevels; ++m) tl.lev[m] = table->lev[m];
     const cudaError_t err = kBwd[table->bits - 1][static_cast<int>(dtype)](
-        tl, packed, grad_out, grad_in, n, static_cast<cudaStream_t>(stream));
+        tl, packed, grad_out, grad_in, n, access_flags(grad_out, grad_in, nullptr, packed, table->bits), static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) { t_last_cuda_error = static_cast<int>(err); return FEWBIT_ERR_CUDA; }
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    return FEWBIT_OK;
+}
+
+fewbit_status fewbit_set_option(fewbit_option opt, int value) {
+    using namespace fewbit;
+    bool ok = false;
+    switch (opt) {
+    case FEWBIT_OPT_FWD_TABLE: ok = value >= 0 && value <= 2; break;
+    case FEWBIT_OPT_FWD_QUEUE: ok = value == 0 || value == 1; break;
+    case FEWBIT_OPT_FWD_ITERS: ok = value >= 0 && value <= 64; break;
+    case FEWBIT_OPT_FWD_WARPS: ok = value >= 0 && value <= 16; break;
+    case FEWBIT_OPT_PDL: ok = value == 0 || value == 1; break;
+    case FEWBIT_OPT_COUNT_TAILS: ok = value == 0 || value == 1; break;
+    default: break;
+    }
+    if (!ok) return FEWBIT_ERR_INVALID_ARG;
+    g_option[opt].store(value, std::memory_order_relaxed);
+    return FEWBIT_OK;
+}
+
+int fewbit_get_option(fewbit_option opt) {
+    return (static_cast<int>(opt) >= 0 && static_cast<int>(opt) < fewbit::kNumOptions) ? fewbit::option(opt) : -1;
+}
+
+fewbit_status fewbit_tail_warp_count(uint64_t *count, int reset) {
+    using namespace fewbit;
+    if (count == nullptr) return FEWBIT_ERR_INVALID_ARG;
+    const cudaError_t err = tail_counter_read(count, reset != 0);
+    if (err != cudaSuccess) { t_last_cuda_error = static_cast<int>(err); return FEWBIT_ERR_CUDA; }
     return FEWBIT_OK;
 }
 

@@ -23,7 +23,8 @@ constexpr int kMaxDevices = 64;
 constexpr size_t kSetWords = static_cast<size_t>(kQueues) * kQueueStride;
 
 // In host code this name is only a handle for the runtime, never a device address.
-static __device__ __align__(256) uint32_t g_counters[kQueueSlots * kSetWords];
+// The word behind the last set is the diagnostic tail counter.
+static __device__ __align__(256) uint32_t g_counters[kQueueSlots * kSetWords + kQueueStride];
 
 struct Slot {
     cudaEvent_t done = nullptr;          // recorded after the last launch that used the set
@@ -38,7 +39,48 @@ struct DeviceState {
 DeviceState g_state[kMaxDevices];
 std::mutex g_mutex;
 
+// Device address of g_counters on the current device (resolved once per device, under g_mutex).
+cudaError_t counters_base(int *dev_out, uint32_t **base) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    DeviceState &st = g_state[dev];
+    if (st.base == nullptr) {
+        void *p = nullptr;
+        err = cudaGetSymbolAddress(&p, g_counters);        // with `dev` current: that device's copy
+        if (err != cudaSuccess) return err;
+        st.base = static_cast<uint32_t *>(p);
+    }
+    *dev_out = dev;
+    *base = st.base;
+    return cudaSuccess;
+}
+
 }  // namespace
+
+cudaError_t tail_counter_address(unsigned int **out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int dev = 0;
+    uint32_t *base = nullptr;
+    const cudaError_t err = counters_base(&dev, &base);
+    if (err != cudaSuccess) return err;
+    *out = base + static_cast<size_t>(kQueueSlots) * kSetWords;
+    return cudaSuccess;
+}
+
+cudaError_t tail_counter_read(uint64_t *count, bool reset) {
+    unsigned int *p = nullptr;
+    cudaError_t err = tail_counter_address(&p);
+    if (err != cudaSuccess) return err;
+    err = cudaDeviceSynchronize();
+    if (err != cudaSuccess) return err;
+    unsigned int v = 0;
+    err = cudaMemcpy(&v, p, sizeof(v), cudaMemcpyDeviceToHost);
+    if (err != cudaSuccess) return err;
+    *count = v;
+    return reset ? cudaMemset(p, 0, sizeof(v)) : cudaSuccess;
+}
 
 cudaError_t queue_acquire(cudaStream_t stream, QueueLease *lease) {
     *lease = QueueLease{};
@@ -49,19 +91,23 @@ cudaError_t queue_acquire(cudaStream_t stream, QueueLease *lease) {
     unsigned long long id = 0;
     err = cudaStreamGetId(stream, &id);
     if (err != cudaSuccess) return err;
-    int dev = 0;
-    err = cudaGetDevice(&dev);
+    // Another host thread may be capturing a stream in the global capture mode, under which an event
+    // query or creation from any thread is refused and would invalidate that capture: what follows
+    // runs in the relaxed mode, which exempts this thread (none of it touches a capturing stream).
+    cudaStreamCaptureMode mode = cudaStreamCaptureModeRelaxed;
+    err = cudaThreadExchangeStreamCaptureMode(&mode);
     if (err != cudaSuccess) return err;
-    if (dev < 0 || dev >= kMaxDevices) return cudaSuccess;
-
+    struct Restore {
+        cudaStreamCaptureMode m;
+        ~Restore() { cudaThreadExchangeStreamCaptureMode(&m); }
+    } restore{mode};
     std::lock_guard<std::mutex> lock(g_mutex);
+    int dev = 0;
+    uint32_t *base = nullptr;
+    err = counters_base(&dev, &base);
+    if (err == cudaErrorInvalidDevice) return cudaSuccess;  // more devices than the table holds: static partition
+    if (err != cudaSuccess) return err;
     DeviceState &st = g_state[dev];
-    if (st.base == nullptr) {
-        void *p = nullptr;
-        err = cudaGetSymbolAddress(&p, g_counters);        // with `dev` current: that device's copy
-        if (err != cudaSuccess) return err;
-        st.base = static_cast<uint32_t *>(p);
-    }
     int pick = -1;
     for (int i = 0; i < kQueueSlots && pick < 0; ++i)       // 1. last used by this stream: ordered behind that use
         if (!st.slot[i].leased && st.slot[i].used && st.slot[i].stream_id == id) pick = i;

@@ -6,7 +6,6 @@ dtype of the exactly rounded binary64 value.  Both sides use the SAME table
 (read back from the library with fewbit_table_get), so the comparison isolates
 the hot path; the solver is compared with the oracle's DP in the CPU tests.
 """
-import os
 from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
@@ -255,7 +254,7 @@ def test_shards_cut_by_shard_range_concatenate_to_the_single_launch_stream():
 
 
 @pytest.mark.parametrize("seed", [1, 2, 3])
-def test_randomised_tables_sizes_dtypes_under_every_variant(seed, monkeypatch):
+def test_randomised_tables_sizes_dtypes_under_every_variant(seed):
     """Random activation, bit width, dtype, size (ragged, whole warp-blocks, several waves), built-in
     or injected tables (random boundaries, duplicates, tiny and large scales), inputs with zeros,
     infinities, NaNs and subnormals: every bucketize variant (search, table with dynamic and with
@@ -285,11 +284,11 @@ def test_randomised_tables_sizes_dtypes_under_every_variant(seed, monkeypatch):
         want = torch.where(torch.isnan(x.float()), torch.zeros_like(want), want)
         outs = []
         for mode, queue in (("never", None), ("always", None), ("always", "never"), ("auto", None)):
-            monkeypatch.setenv("FEWBIT_FWD_TABLE", mode)
+            fb.fewbit_set_option("fwd_table", mode)
             if queue:
-                monkeypatch.setenv("FEWBIT_FWD_QUEUE", queue)
+                fb.fewbit_set_option("fwd_queue", queue)
             else:
-                monkeypatch.delenv("FEWBIT_FWD_QUEUE", raising=False)
+                fb.fewbit_set_option("fwd_queue", "auto")
             outs.append(fb.fewbit_fwd(t, x))
         torch.cuda.synchronize()
         what = (seed, dtype, act, bits, n)
@@ -299,7 +298,7 @@ def test_randomised_tables_sizes_dtypes_under_every_variant(seed, monkeypatch):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
-def test_degenerate_boundary_tables(dtype, monkeypatch):
+def test_degenerate_boundary_tables(dtype):
     """Injected tables at the edges of what Eq. 2 allows: all boundaries equal, infinite boundaries,
     boundaries at the smallest subnormal, at +-0 and beyond the binary16 range; inputs with zeros,
     infinities, NaN, subnormals and the largest finite values.  Codes are torch.bucketize's under
@@ -323,11 +322,11 @@ def test_degenerate_boundary_tables(dtype, monkeypatch):
                 want = torch.bucketize(x.float(), edges, right=False)
                 want = torch.where(torch.isnan(x.float()), torch.zeros_like(want), want)
                 for mode, queue in (("never", None), ("always", None), ("always", "never")):
-                    monkeypatch.setenv("FEWBIT_FWD_TABLE", mode)
+                    fb.fewbit_set_option("fwd_table", mode)
                     if queue:
-                        monkeypatch.setenv("FEWBIT_FWD_QUEUE", queue)
+                        fb.fewbit_set_option("fwd_queue", queue)
                     else:
-                        monkeypatch.delenv("FEWBIT_FWD_QUEUE", raising=False)
+                        fb.fewbit_set_option("fwd_queue", "auto")
                     _, pk = fb.fewbit_fwd(t, x)
                     assert torch.equal(_unpack_on_device(pk, bits, n), want), (dtype, bits, s, n, mode, queue)
 
@@ -359,7 +358,7 @@ def test_backward_with_special_levels_and_gradients(dtype):
 
 
 @pytest.mark.parametrize("seed", [6, 7])
-def test_randomised_folded_tables_under_every_variant(seed, monkeypatch):
+def test_randomised_folded_tables_under_every_variant(seed):
     """Folded tables (caption of Fig. 3) with random range and grid, random dtype, size and input
     scale: the codes are torch.bucketize's of |x| (NaN -> 0), the same under every bucketize variant,
     and the backward product is torch's binary32 product rounded once."""
@@ -379,11 +378,11 @@ def test_randomised_folded_tables_under_every_variant(seed, monkeypatch):
         want = torch.where(torch.isnan(x.float()), torch.zeros_like(want), want)
         outs = []
         for mode, queue in (("never", None), ("always", None), ("always", "never"), ("auto", None)):
-            monkeypatch.setenv("FEWBIT_FWD_TABLE", mode)
+            fb.fewbit_set_option("fwd_table", mode)
             if queue:
-                monkeypatch.setenv("FEWBIT_FWD_QUEUE", queue)
+                fb.fewbit_set_option("fwd_queue", queue)
             else:
-                monkeypatch.delenv("FEWBIT_FWD_QUEUE", raising=False)
+                fb.fewbit_set_option("fwd_queue", "auto")
             outs.append(fb.fewbit_fwd(t, x))
         torch.cuda.synchronize()
         what = (seed, dtype, act, bits, n)
@@ -396,7 +395,7 @@ def test_randomised_folded_tables_under_every_variant(seed, monkeypatch):
 
 
 @pytest.mark.parametrize("seed", [4, 5])
-def test_randomised_backward_and_bias_against_torch_arithmetic(seed, monkeypatch):
+def test_randomised_backward_and_bias_against_torch_arithmetic(seed):
     """Random sizes, dtypes, activations and bit widths: grad_in equals torch's binary32 product
     rounded once, and f(x + bias) equals the plain forward on torch's binary32 sum rounded once."""
     import random
@@ -419,12 +418,12 @@ def test_randomised_backward_and_bias_against_torch_arithmetic(seed, monkeypatch
         b = torch.randn(cols, device=DEV).to(TORCH_DT[dtype])
         z = (xb.float() + b.float()[None, :]).to(TORCH_DT[dtype])
         for mode in ("never", "always"):
-            monkeypatch.setenv("FEWBIT_FWD_TABLE", mode)
+            fb.fewbit_set_option("fwd_table", mode)
             y1, p1 = fb.fewbit_fwd_bias(t, xb, b)
             y2, p2 = fb.fewbit_fwd(t, z)
             torch.cuda.synchronize()
             assert torch.equal(p1, p2) and torch.equal(y1.view(torch.uint8), y2.view(torch.uint8)), (seed, dtype, act, bits, rows, cols, mode)
-        monkeypatch.delenv("FEWBIT_FWD_TABLE")
+        fb.fewbit_set_option("fwd_table", "auto")
 
 
 # --------------------------------------------------------------------------
@@ -600,13 +599,9 @@ def test_more_than_2_to_the_32_elements():
 def table_mode(request):
     """Runs a test under each bucketize variant: size-based choice, shared-memory
     code table forced on (where the table has one), forced off."""
-    old = os.environ.get("FEWBIT_FWD_TABLE")
-    os.environ["FEWBIT_FWD_TABLE"] = request.param
+    fb.fewbit_set_option("fwd_table", request.param)
     yield request.param
-    if old is None:
-        os.environ.pop("FEWBIT_FWD_TABLE", None)
-    else:
-        os.environ["FEWBIT_FWD_TABLE"] = old
+    fb.fewbit_set_option("fwd_table", "auto")
 
 
 
@@ -767,8 +762,165 @@ def test_misaligned_device_buffers_are_rejected():
     t = table("gelu", 2)
     x = torch.zeros(4096 + 8, device=DEV)
     with pytest.raises(fb.FewbitError) as e:
-        fb.fewbit_fwd(t, x[1:4097])
+        fb.fewbit_fwd(t, x[1:4097])                       # 4 bytes off: below the 16-byte rule
     assert e.value.status == 3
+    with pytest.raises(fb.FewbitError) as e:
+        fb.fewbit_fwd(t, x[2:4098])
+    assert e.value.status == 3
+    h = torch.zeros(4096 + 8, device=DEV, dtype=torch.bfloat16)
+    with pytest.raises(fb.FewbitError) as e:
+        fb.fewbit_fwd(t, h[4:4100])                       # 8 bytes off
+    assert e.value.status == 3
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16", "f32"])
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+def test_buffers_at_the_minimum_alignment(dtype, bits, table_mode):
+    """The rule of the boundary: element buffers 16-byte aligned, packed words 4-byte aligned.  Every
+    buffer is a view that starts 16 bytes (elements) or 4, 8, 12 bytes (packed) into a 256-byte aligned
+    allocation, with canaries on both sides; codes and grad_in bit-exact with the oracle, y within 2 ulp.
+    Sizes cover the ragged path alone, whole warp-blocks and the table variants' sizes."""
+    tdt = TORCH_DT[dtype]
+    es = torch.empty(0, dtype=tdt).element_size()
+    off = 16 // es
+    gen = torch.Generator(device=DEV).manual_seed(17 + bits)
+    t = table("sigmoid", bits)
+    for n, poff in ((1000, 1), (5 * 1024 + 77, 2), ((1 << 22) + 1024 * 3 + 5, 3), ((1 << 23) + 9, 1)):
+        words = fb.fewbit_packed_bytes(n, bits) // 4
+        x = (torch.randn(n + off, generator=gen, device=DEV) * 2).to(tdt)[off:]
+        g = torch.randn(n + off, generator=gen, device=DEV).to(tdt)[off:]
+        ybuf = torch.full((n + 2 * 128 + off,), 777.0, dtype=tdt, device=DEV)
+        gbuf = torch.full((n + 2 * 128 + off,), 777.0, dtype=tdt, device=DEV)
+        pbuf = torch.full((words + 2 * 64 + poff,), 0x5A5A5A5A, dtype=torch.int32, device=DEV)
+        y, gi, pk = ybuf[128 + off:128 + off + n], gbuf[128 + off:128 + off + n], pbuf[64 + poff:64 + poff + words]
+        assert x.data_ptr() % 32 == 16 and y.data_ptr() % 32 == 16 and pk.data_ptr() % 16 == 4 * poff
+        fb.fewbit_fwd(t, x, y, pk)
+        fb.fewbit_bwd(t, pk, g, gi)
+        torch.cuda.synchronize()
+        for buf, lo, m, fill in ((ybuf, 128 + off, n, 777.0), (gbuf, 128 + off, n, 777.0), (pbuf, 64 + poff, words, 0x5A5A5A5A)):
+            assert bool((buf[:lo] == fill).all()) and bool((buf[lo + m:] == fill).all()), "wrote outside the buffer"
+        compare_full("sigmoid", bits, x, g, y, pk, gi, f"min alignment {dtype} k={bits} n={n}")
+        # the same call with the bias in front, the bias view 16 bytes in as well
+        cols = 8 * 25
+        rows = n // cols
+        if rows:
+            m = rows * cols
+            b = torch.randn(cols + off, generator=gen, device=DEV).to(tdt)[off:]
+            z = (x[:m].float().view(rows, cols) + b.float()[None, :]).to(tdt).reshape(-1)
+            fb.fewbit_fwd_bias(t, x[:m].view(rows, cols), b, y[:m].view(rows, cols), pk)
+            y2, p2 = fb.fewbit_fwd(t, z.contiguous())
+            torch.cuda.synchronize()
+            mw = fb.fewbit_packed_bytes(m, bits) // 4
+            assert torch.equal(pk[:mw], p2) and torch.equal(y[:m].view(torch.uint8), y2.view(torch.uint8))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_shards_cut_on_32_elements(dtype):
+    """A flat tensor cut on multiples of 32 elements: each shard's x, y and packed views satisfy the
+    alignment rule as they are, and the shards written side by side into ONE y and ONE packed buffer
+    are the single-launch result."""
+    tdt = TORCH_DT[dtype]
+    n = (1 << 21) + 32 * 37 + 11
+    x = (torch.randn(n, device=DEV) * 1.5).to(tdt)
+    g = torch.randn(n, device=DEV).to(tdt)
+    for bits in (1, 2, 3, 4):
+        t = table("gelu", bits)
+        y, pk = fb.fewbit_fwd(t, x)
+        gi = fb.fewbit_bwd(t, pk, g)
+        for world in (3, 7):
+            y2, p2, gi2 = torch.zeros_like(y), torch.zeros_like(pk), torch.zeros_like(gi)
+            for rank in range(world):
+                lo, hi = wl.shard_range(n, rank, world, align=32)
+                assert lo % 32 == 0
+                w0, w1 = lo // 32 * bits, fb.fewbit_packed_bytes(hi, bits) // 4
+                fb.fewbit_fwd(t, x[lo:hi], y2[lo:hi], p2[w0:w1])
+                fb.fewbit_bwd(t, p2[w0:w1], g[lo:hi], gi2[lo:hi])
+            torch.cuda.synchronize()
+            assert torch.equal(p2, pk), (dtype, bits, world)
+            assert torch.equal(y2.view(torch.uint8), y.view(torch.uint8))
+            assert torch.equal(gi2.view(torch.uint8), gi.view(torch.uint8))
+
+
+# --------------------------------------------------------------------------
+# the ragged tail has exactly one owner, also in place
+# --------------------------------------------------------------------------
+def _tail_sizes():
+    # n = k * 1024 + 5: the partial warp-block sits at every offset 0 .. 11 of a 12-warp CTA (and of
+    # 4-warp ones); 2^24 + 7 is the sweep's ragged size
+    return [k * 1024 + 5 for k in range(60, 72)] + [2 ** 24 + 7]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("bits", [3, 4])
+def test_ragged_tail_has_one_owner_and_works_in_place(dtype, bits):
+    """y == x with a ragged last warp-block, binary32 and bfloat16, code table forced and size-based,
+    static and dynamic partition, CTA widths of 4, 12 and 16 warps: exactly one warp runs the tail
+    (counted on the device), and codes, y and grad_in are the oracle's."""
+    tdt = TORCH_DT[dtype]
+    gen = torch.Generator(device=DEV).manual_seed(3 + bits)
+    fb.fewbit_set_option("count_tails", 1)
+    fb.fewbit_tail_warp_count(reset=True)
+    for act in ("leaky_relu", "sigmoid"):
+        t = table(act, bits)
+        for n in _tail_sizes():
+            x = (torch.randn(n, generator=gen, device=DEV) * 2).to(tdt)
+            g = torch.randn(n, generator=gen, device=DEV).to(tdt)
+            ref = None
+            for mode, queue, iters in (("auto", "auto", 0), ("always", "never", 0), ("always", "auto", 0), ("always", "never", 1),
+                                       ("always", "never", 3), ("never", "auto", 0), ("never", "auto", 2)):
+                fb.fewbit_set_option("fwd_table", mode)
+                fb.fewbit_set_option("fwd_queue", queue)
+                fb.fewbit_set_option("fwd_iters", iters)
+                y = x.clone()
+                pk = torch.full((fb.fewbit_packed_bytes(n, bits) // 4,), 0x5A5A5A5A, dtype=torch.int32, device=DEV)
+                fb.fewbit_fwd(t, y, y, pk)                      # in place
+                assert fb.fewbit_tail_warp_count(reset=True) == 1, (dtype, bits, act, n, mode, queue, iters)
+                if ref is None:
+                    gi = g.clone()
+                    fb.fewbit_bwd(t, pk, gi, gi)
+                    torch.cuda.synchronize()
+                    if n < 2 ** 20:
+                        compare_full(act, bits, x, g, y, pk, gi, f"in place, ragged, n={n}")
+                    else:
+                        compare_sampled(act, bits, x, g, y, pk, gi, f"in place, ragged, n={n}", blocks=8, block_elems=4096)
+                    ref = (y, pk)
+                else:
+                    assert torch.equal(pk, ref[1]) and torch.equal(y.view(torch.uint8), ref[0].view(torch.uint8)), \
+                        (dtype, bits, act, n, mode, queue, iters)
+            # the same sizes through the bias entry point (rows of 8 elements need n % 8 == 0: cut the view)
+            m = n // 8 * 8
+            b = torch.zeros(8, device=DEV, dtype=tdt)
+            fb.fewbit_set_option("fwd_table", "always")
+            fb.fewbit_set_option("fwd_queue", "never")
+            fb.fewbit_set_option("fwd_iters", 0)
+            yb = x[:m].clone().view(-1, 8)
+            pb = torch.empty(fb.fewbit_packed_bytes(m, bits) // 4, dtype=torch.int32, device=DEV)
+            fb.fewbit_fwd_bias(t, yb, b, yb, pb)
+            assert fb.fewbit_tail_warp_count(reset=True) == (1 if m % 1024 else 0)
+            y0, p0 = fb.fewbit_fwd(t, x[:m].contiguous())
+            assert fb.fewbit_tail_warp_count(reset=True) == (1 if m % 1024 else 0)
+            torch.cuda.synchronize()
+            assert torch.equal(pb, p0) and torch.equal(yb.view(torch.uint8).reshape(-1), y0.view(torch.uint8).reshape(-1))
+
+
+@pytest.mark.parametrize("warps,iters", [(1, 0), (2, 5), (0, 1), (0, 64), (16, 2), (3, 0)])
+def test_launch_geometry_overrides_do_not_change_the_result(warps, iters):
+    """FEWBIT_OPT_FWD_WARPS / FEWBIT_OPT_FWD_ITERS only reshape the grid (a single-warp CTA included):
+    same y and packed words as the default launch, bfloat16 at 4 bits (shared threshold-pair table)
+    and binary32."""
+    for dtype, act, bits in (("bf16", "silu", 4), ("bf16", "gelu", 3), ("f32", "tanh", 4), ("f16", "elu", 4)):
+        t = table(act, bits)
+        for n in (70001, (1 << 21) + 1029):
+            x = (torch.randn(n, device=DEV) * 2).to(TORCH_DT[dtype])
+            fb.fewbit_set_option("fwd_table", "never")
+            y0, p0 = fb.fewbit_fwd(t, x)
+            fb.fewbit_set_option("fwd_warps", warps)
+            fb.fewbit_set_option("fwd_iters", iters)
+            y1, p1 = fb.fewbit_fwd(t, x)
+            fb.fewbit_set_option("fwd_warps", 0)
+            fb.fewbit_set_option("fwd_iters", 0)
+            torch.cuda.synchronize()
+            assert torch.equal(p0, p1) and torch.equal(y0.view(torch.uint8), y1.view(torch.uint8)), (dtype, act, bits, n)
 
 
 def test_runs_on_a_side_stream():
@@ -785,7 +937,7 @@ def test_runs_on_a_side_stream():
 
 
 @pytest.mark.parametrize("bits", [3, 4])
-def test_dynamic_table_variant_on_concurrent_streams(bits, monkeypatch):
+def test_dynamic_table_variant_on_concurrent_streams(bits):
     """The table variant of the 16-bit types hands out warp-blocks through leased work counters.
     Three streams at once, twice each (a stream reuses its own counters, different streams must
     not share any): every launch gives exactly what the search variant gives on the same input,
@@ -794,12 +946,12 @@ def test_dynamic_table_variant_on_concurrent_streams(bits, monkeypatch):
     t = table("gelu", bits)
     gen = torch.Generator(device=DEV).manual_seed(31 + bits)
     xs = [torch.randn(n, device=DEV, generator=gen).bfloat16() for _ in range(3)]
-    monkeypatch.setenv("FEWBIT_FWD_TABLE", "never")
+    fb.fewbit_set_option("fwd_table", "never")
     refs = [fb.fewbit_fwd(t, x) for x in xs]
     torch.cuda.synchronize()
     g = torch.ones(n, device=DEV).bfloat16()
     compare_sampled("gelu", bits, xs[0], g, refs[0][0], refs[0][1], fb.fewbit_bwd(t, refs[0][1], g), "search variant")
-    monkeypatch.setenv("FEWBIT_FWD_TABLE", "always")
+    fb.fewbit_set_option("fwd_table", "always")
     streams = [torch.cuda.Stream() for _ in xs]
     outs = []
     for rep in range(2):
@@ -816,35 +968,35 @@ def test_dynamic_table_variant_on_concurrent_streams(bits, monkeypatch):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
-def test_dynamic_and_static_partition_agree_on_whole_arrays(dtype, monkeypatch):
+def test_dynamic_and_static_partition_agree_on_whole_arrays(dtype):
     """Every element and every packed word of the dynamically distributed table variant equals the
     statically partitioned one (a warp-block dropped or done twice would show), ragged tail included."""
     n = (1 << 24) + 4097
     x = (torch.randn(n, device=DEV) * 2).to(TORCH_DT[dtype])
-    monkeypatch.setenv("FEWBIT_FWD_TABLE", "always")
+    fb.fewbit_set_option("fwd_table", "always")
     for act in ("sigmoid", "gelu"):
         for bits in (3, 4):
             t = table(act, bits)
-            monkeypatch.setenv("FEWBIT_FWD_QUEUE", "never")
+            fb.fewbit_set_option("fwd_queue", "never")
             y0, p0 = fb.fewbit_fwd(t, x)
-            monkeypatch.delenv("FEWBIT_FWD_QUEUE")
+            fb.fewbit_set_option("fwd_queue", "auto")
             y1, p1 = fb.fewbit_fwd(t, x)
             torch.cuda.synchronize()
             assert torch.equal(p0, p1), (dtype, act, bits)
             assert torch.equal(y0.view(torch.uint8), y1.view(torch.uint8)), (dtype, act, bits)
 
 
-def test_more_streams_than_work_counter_sets_from_several_host_threads(monkeypatch):
+def test_more_streams_than_work_counter_sets_from_several_host_threads():
     """24 streams driven by 6 host threads, two table-variant launches each, nothing waited for in
     between: more launches in flight than there are sets of work counters, so some take the static
     partition.  Every result equals the search variant's."""
     n = (1 << 23) + 1024 * 5 + 3
     t = table("gelu", 4)
     x = torch.randn(n, device=DEV).mul_(1.7).bfloat16()
-    monkeypatch.setenv("FEWBIT_FWD_TABLE", "never")
+    fb.fewbit_set_option("fwd_table", "never")
     y_ref, p_ref = fb.fewbit_fwd(t, x)
     torch.cuda.synchronize()
-    monkeypatch.setenv("FEWBIT_FWD_TABLE", "always")
+    fb.fewbit_set_option("fwd_table", "always")
     streams = [torch.cuda.Stream() for _ in range(24)]
     outs = [None] * 48
 

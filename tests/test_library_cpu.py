@@ -119,13 +119,17 @@ def test_hot_path_argument_checks_need_no_gpu(lib):
     assert lib.fewbit_fwd(h, None, A, A, 10, 0, None) == 1
     assert lib.fewbit_fwd(h, A, None, A, 10, 0, None) == 1
     assert lib.fewbit_fwd(h, A, A, None, 10, 0, None) == 1
-    assert lib.fewbit_fwd(h, A + 16, A, A, 10, 0, None) == 3
+    # the rule: element buffers 16-byte aligned, packed words 4-byte aligned (any dtype)
+    assert lib.fewbit_fwd(h, A + 8, A, A, 10, 0, None) == 3
     assert lib.fewbit_fwd(h, A, A + 8, A, 10, 1, None) == 3
-    assert lib.fewbit_fwd(h, A, A, A + 4, 10, 1, None) == 3
+    assert lib.fewbit_fwd(h, A, A, A + 2, 10, 1, None) == 3
+    assert lib.fewbit_fwd(h, A, A + 4, A, 10, 2, None) == 3
     assert lib.fewbit_fwd(h, None, None, None, 0, 0, None) == 0
     assert lib.fewbit_bwd(None, A, A, A, 10, 0, None) == 1
     assert lib.fewbit_bwd(h, None, A, A, 10, 0, None) == 1
     assert lib.fewbit_bwd(h, A, A + 2, A, 10, 1, None) == 3
+    assert lib.fewbit_bwd(h, A, A, A + 8, 10, 0, None) == 3
+    assert lib.fewbit_bwd(h, A + 1, A, A, 10, 0, None) == 3
     assert lib.fewbit_bwd(h, A, A, A, 0, 1, None) == 0
     assert lib.fewbit_fwd_host(h, A, A, A, 10, 0, None, 0) == 1
     assert lib.fewbit_fwd_host(h, A, A, A, 10, 0, A, 16) == 5
@@ -136,11 +140,21 @@ def test_hot_path_argument_checks_need_no_gpu(lib):
     assert lib.fewbit_fwd_bias(h, A, None, A, A, 4, 1024, 1, None) == 1
     assert lib.fewbit_fwd_bias(h, A, A, A, A, 4, 1020, 1, None) == 2         # a row is not a whole number of 8-element chunks
     assert lib.fewbit_fwd_bias(h, A, A, A, A, 4, 1 << 32, 1, None) == 2       # row length beyond 32 bits
-    assert lib.fewbit_fwd_bias(h, A, A + 16, A, A, 4, 1024, 1, None) == 3
+    assert lib.fewbit_fwd_bias(h, A, A + 8, A, A, 4, 1024, 1, None) == 3
+    assert lib.fewbit_fwd_bias(h, A, A, A, A + 2, 4, 1024, 1, None) == 3
     assert lib.fewbit_fwd_bias(h, A, A, A, A, 1 << 40, 1 << 30, 1, None) == 1  # rows * cols overflows
     assert lib.fewbit_fwd_bias(h, None, None, None, None, 0, 1024, 1, None) == 0
     tf = fb.fewbit_table_create_folded("tanh", 2)
     assert lib.fewbit_fwd_bias(tf.handle, A, A, A, A, 4, 1024, 1, None) == 2  # no folded tables with a bias
+    # options: unknown option / value out of range are refused, valid ones read back
+    assert lib.fewbit_set_option(99, 0) == 1 and lib.fewbit_get_option(99) == -1
+    assert lib.fewbit_set_option(0, 3) == 1 and lib.fewbit_set_option(2, -1) == 1 and lib.fewbit_set_option(2, 65) == 1
+    assert lib.fewbit_set_option(3, 17) == 1 and lib.fewbit_set_option(4, 2) == 1
+    for opt, default, other in ((0, 0, 2), (1, 0, 1), (2, 0, 7), (3, 0, 4), (4, 1, 0), (5, 0, 1)):
+        assert lib.fewbit_get_option(opt) == default
+        assert lib.fewbit_set_option(opt, other) == 0 and lib.fewbit_get_option(opt) == other
+        assert lib.fewbit_set_option(opt, default) == 0
+    assert lib.fewbit_tail_warp_count(None, 0) == 1
     # the accuracy scan: act, first pattern, count, result
     assert lib.fewbit_f32_activation_scan(99, 0, 16, A, None) == 1
     assert lib.fewbit_f32_activation_scan(0, 0, 16, None, None) == 1

@@ -33,6 +33,12 @@ def test_shard_ranges_tile_and_align():
                 assert hi % 128 == 0 or hi == n
     with pytest.raises(ValueError):
         wl.shard_range(10, 2, 2)
+    # cuts on 32 elements (the unit the library's alignment rule allows): whole packed words for every width
+    for n in (31, 32, 33, 2 ** 24 + 7):
+        for world in (2, 5, 8):
+            cuts = [wl.shard_range(n, r, world, align=32) for r in range(world)]
+            assert cuts[0][0] == 0 and cuts[-1][1] == n and all(b == c for (_, b), (c, _) in zip(cuts, cuts[1:]))
+            assert all(lo % 32 == 0 for lo, _ in cuts)
 
 
 def _free_port():
@@ -83,3 +89,21 @@ def test_two_gloo_ranks_reproduce_the_single_stream(tmp_path, bits):
     world, n = 2, 100000 + 37
     mp.spawn(_worker, args=(world, _free_port(), n, bits, str(tmp_path)), nprocs=world, join=True)
     assert os.path.exists(tmp_path / "ok")
+
+
+def test_bench_starts_its_own_ranks_when_asked_for_more_than_one_gpu():
+    """`python bench.py --gpus 2` started plainly (no torchrun) re-launches itself as two ranks on
+    127.0.0.1.  Checked with the reference arm, which needs no GPU: rank 0 alone prints the line, and
+    the line reports the two ranks."""
+    import json
+    import subprocess
+    import sys
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "reference", "--steps", "1",
+                          "--warmup", "0", "--ref-sample", "65536"], capture_output=True, text=True, env=env, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(ln) for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2 and lines[0]["ranks_started"] == 2
