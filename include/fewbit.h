@@ -261,8 +261,9 @@ FEWBIT_API size_t fewbit_host_workspace_bytes(size_t chunk_elems, fewbit_dtype d
  * results as fewbit_fwd.  The tensor is cut into chunks; each chunk is copied
  * to `workspace` (DEVICE, caller-owned, 256-byte aligned, `workspace_bytes`
  * long), run through the forward kernel and copied back, with the copies of
- * neighbouring chunks overlapping the kernel on three internal streams.
- * Blocks until the results are in host memory.  Page-locked host buffers are
+ * neighbouring chunks overlapping the kernel on three internal streams (created
+ * by the first call on a device and kept for later calls; concurrent calls get
+ * triples of their own).  Blocks until the results are in host memory.  Page-locked host buffers are
  * needed for the copies to overlap; pageable ones work, slower.
  * FEWBIT_ERR_ALLOC if the workspace cannot hold one 1024-element chunk.
  * Calls on the same device that overlap in time must use disjoint workspaces.
@@ -298,11 +299,19 @@ FEWBIT_API fewbit_status fewbit_bwd_host(const fewbit_table *table, const uint32
  * the call returns.  n > fewbit_static_max_elements() is rejected with
  * FEWBIT_ERR_TOO_LARGE (split the tensor on a multiple of 1024 elements and
  * call once per piece, or use fewbit_fwd_host).  The call makes no
- * cudaMalloc / cudaFree and creates no stream or event.
+ * cudaMalloc / cudaFree and, with the default options, creates no stream or
+ * event (at this capacity the kernel variants that lease work counters are
+ * never the size-based choice).
  *
  * The first call on each device looks up the device address of the array
  * (cudaGetSymbolAddress, with that device current); make that first call
- * outside of any stream capture.  All calls on a device share the one array:
+ * outside of any stream capture.  Under CUDA's lazy module loading that same
+ * first call is what loads the part of the library holding the array, i.e. it
+ * is the moment the ~2.1 MiB are taken from the device: a caller whose pool
+ * later claims all device memory should make one (small) call at start-up,
+ * before the pool does, or run with CUDA_MODULE_LOADING=EAGER.  The address is
+ * cached per device for the life of the process; it does not survive a
+ * cudaDeviceReset.  All calls on a device share the one array:
  * it still holds the previous call's data (harmless -- every byte that is
  * read is written first, so nothing needs clearing), and two calls whose GPU
  * work overlaps in time, from different threads or streams, race on it.

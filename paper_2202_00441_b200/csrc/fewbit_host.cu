@@ -2,11 +2,14 @@
 // host memory.  The tensor is streamed through a caller-owned device
 // workspace in chunks; chunk c uses pipeline stage c % 3, each stage has its
 // own stream, so the host->device copy of one chunk, the kernel of the
-// previous one and the device->host copy of the one before overlap.
+// previous one and the device->host copy of the one before overlap.  The
+// streams are created on first use and reused by later calls.
 #include <cuda_runtime.h>
 
 #include <algorithm>
 #include <cstdint>
+#include <mutex>
+#include <vector>
 
 #include "fewbit_internal.h"
 
@@ -25,18 +28,51 @@ inline size_t stage_bytes(size_t chunk, fewbit_dtype d, int bits) {
     return 2 * round_up(chunk * elem_bytes(d), kSlotAlign) + round_up(chunk * bits / 8, kSlotAlign);
 }
 
+// The three non-blocking streams of one call.  They are created once and kept: a call takes a free
+// triple of the current device from a small per-device pool (or creates one when all are in use by
+// concurrent calls of other host threads) and hands it back when it returns; nothing is destroyed
+// before the process ends.  A call only returns after its streams have drained, so a triple taken
+// from the pool is idle.
+constexpr int kMaxDevices = 64;
+struct StreamTriple { cudaStream_t s[kStages] = {nullptr, nullptr, nullptr}; };
+std::mutex g_pool_mutex;
+std::vector<StreamTriple> g_pool[kMaxDevices];
+
 struct Pipeline {
     cudaStream_t stream[kStages] = {nullptr, nullptr, nullptr};
     cudaError_t err = cudaSuccess;
+    int dev = -1;
+    bool pooled = false;
     bool ok(cudaError_t e) { if (e != cudaSuccess && err == cudaSuccess) err = e; return e == cudaSuccess; }
     bool open() {
+        if (!ok(cudaGetDevice(&dev))) return false;
+        pooled = dev >= 0 && dev < kMaxDevices;
+        if (pooled) {
+            std::lock_guard<std::mutex> lock(g_pool_mutex);
+            if (!g_pool[dev].empty()) {
+                for (int s = 0; s < kStages; ++s) stream[s] = g_pool[dev].back().s[s];
+                g_pool[dev].pop_back();
+                return true;
+            }
+        }
         for (int s = 0; s < kStages; ++s)
             if (!ok(cudaStreamCreateWithFlags(&stream[s], cudaStreamNonBlocking))) return false;
         return true;
     }
     void close() {
+        bool complete = true;
+        for (int s = 0; s < kStages; ++s) {
+            if (stream[s]) ok(cudaStreamSynchronize(stream[s])); else complete = false;
+        }
+        if (pooled && complete) {
+            StreamTriple t;
+            for (int s = 0; s < kStages; ++s) { t.s[s] = stream[s]; stream[s] = nullptr; }
+            std::lock_guard<std::mutex> lock(g_pool_mutex);
+            g_pool[dev].push_back(t);
+            return;
+        }
         for (int s = 0; s < kStages; ++s)
-            if (stream[s]) { ok(cudaStreamSynchronize(stream[s])); cudaStreamDestroy(stream[s]); stream[s] = nullptr; }
+            if (stream[s]) { cudaStreamDestroy(stream[s]); stream[s] = nullptr; }
     }
 };
 

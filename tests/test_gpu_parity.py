@@ -6,6 +6,7 @@ dtype of the exactly rounded binary64 value.  Both sides use the SAME table
 (read back from the library with fewbit_table_get), so the comparison isolates
 the hot path; the solver is compared with the oracle's DP in the CPU tests.
 """
+import os
 from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
@@ -22,7 +23,8 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 GUARD = 64            # guard elements / words placed around every output buffer
 TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
-_POOL = ThreadPoolExecutor(max_workers=8)
+_THREADS = max(1, len(os.sched_getaffinity(0)))
+_POOL = ThreadPoolExecutor(max_workers=_THREADS)
 _TABLES = {}
 
 
@@ -103,6 +105,22 @@ def compare_full(act, bits, x, g, y, packed, gi, what):
     compare_block(act, bits, np_bits(x), np_bits(g), np_bits(y), np_bits(packed).view(np.uint32), np_bits(gi), what)
 
 
+def compare_every_element(act, bits, x, g, y, packed, gi, what):
+    """compare_full for tensors of any size: the arrays go to the host once and are cut into one
+    contiguous shard per host thread (on multiples of 1024 elements, so every shard's packed words are
+    whole); every element of y and grad_in and every packed word is compared with the oracle."""
+    n = x.numel()
+    xn, gn, yn, gin = np_bits(x), np_bits(g), np_bits(y), np_bits(gi)
+    pn = np_bits(packed).view(np.uint32)
+    shards = max(1, min(4 * _THREADS, n // (1 << 20)))
+    jobs = []
+    for r in range(shards):
+        lo, hi = wl.shard_range(n, r, shards, 1024)
+        if hi > lo:
+            jobs.append((lo, xn[lo:hi], gn[lo:hi], yn[lo:hi], pn[lo // 32 * bits:(hi * bits + 31) // 32], gin[lo:hi]))
+    list(_POOL.map(lambda j: compare_block(act, bits, j[1], j[2], j[3], j[4], j[5], f"{what} @ {j[0]}"), jobs))
+
+
 def compare_sampled(act, bits, x, g, y, packed, gi, what, blocks=24, block_elems=8192, seed=0, also_at=()):
     """Element-by-element comparison on randomly placed 32-aligned blocks plus
     the first and the last (ragged) block (and blocks starting at `also_at`)."""
@@ -145,12 +163,12 @@ def test_config2_silu_bf16_full():
         list(_POOL.map(lambda j: compare_block(*j), jobs))
 
 
-def test_config3_gelu_bf16_llm_ffn_sampled():
+def test_config3_gelu_bf16_llm_ffn_every_element():
     x, g = wl.draw(wl.C3, DEV)
     assert x.numel() == 2 ** 28
     for bits in wl.C3.bits:
         y, p, gi = run_gpu("gelu", bits, x, g)
-        compare_sampled("gelu", bits, x, g, y, p, gi, f"c3 k={bits}", blocks=48, seed=bits)
+        compare_every_element("gelu", bits, x, g, y, p, gi, f"c3 k={bits}")
         # every code of the full-size launch against torch.bucketize, 2^26 elements at a time
         s, _ = table("gelu", bits).arrays()
         edges = torch.tensor(s, device=DEV)
@@ -163,11 +181,11 @@ def test_config3_gelu_bf16_llm_ffn_sampled():
         del y, p, gi
 
 
-def test_config4_cnn_f32_sampled():
+def test_config4_cnn_f32_every_element():
     x, g = wl.draw(wl.C4, DEV)
     for act in wl.C4.acts:
         y, p, gi = run_gpu(act, 2, x, g)
-        compare_sampled(act, 2, x, g, y, p, gi, f"c4 {act}", blocks=48, seed=3)
+        compare_every_element(act, 2, x, g, y, p, gi, f"c4 {act}")
 
 
 @pytest.mark.parametrize("n", [2 ** 16, 2 ** 20])
@@ -187,11 +205,17 @@ def test_config5_sweep_large_sampled(n, dtype):
     case = next(c for c in wl.sweep_cases([n]) if c.dtype == dtype)
     x, g = wl.draw(case, DEV)
     blocks = 12 if n < 2 ** 28 else 8
+    # every element for two activations (the heaviest arithmetic and one with an exponential in both
+    # tails), sampled blocks for the others; at 2^24 (+7) every element of all seven
+    everywhere = case.acts if n < 2 ** 28 else ("gelu", "softplus")
     for act in case.acts:
         for bits in case.bits:
             y, p, gi = run_gpu(act, bits, x, g)
-            compare_sampled(act, bits, x, g, y, p, gi, f"c5 {act} k={bits} n={n} {dtype}", blocks=blocks,
-                            block_elems=4096, seed=bits)
+            what = f"c5 {act} k={bits} n={n} {dtype}"
+            if act in everywhere:
+                compare_every_element(act, bits, x, g, y, p, gi, what)
+            else:
+                compare_sampled(act, bits, x, g, y, p, gi, what, blocks=blocks, block_elems=4096, seed=bits)
             del y, p, gi
 
 
@@ -1274,3 +1298,43 @@ def test_f32_scan_agrees_with_the_oracle_on_a_range():
         hist = [int((d == k).sum()) for k in range(3)] + [int((d > 2).sum())]
         r = fb.fewbit_f32_activation_scan(act, first, count)
         assert r["hist"] == hist, (act, r, hist)
+
+
+@pytest.mark.parametrize("act", wl.ACTIVATIONS + wl.EXTRA_ACTIVATIONS)
+def test_f32_scan_reference_is_tied_to_the_oracle_on_every_exponent(act):
+    """The scan over all 2^32 inputs compares the library's binary32 arithmetic with a binary64
+    evaluation ON THE DEVICE.  This ties that reference to the oracle across the whole range: for every
+    binary32 exponent (subnormals included) and both signs, a stretch of 2^13 consecutive mantissas at
+    a random offset plus 2^11 scattered ones go through fewbit_fwd; y is within 2 ulp of the oracle on
+    all of them, and on the stretches the histogram of |y - oracle| in ulps, recomputed on the host,
+    is exactly what the scan reports for the same patterns."""
+    rng = np.random.default_rng(1234 + fb.ACTS[act])
+    stretch, scattered = 1 << 13, 1 << 11
+    firsts, pats = [], []
+    for sign in (0, 1):
+        for e in range(255):                                 # exponent 255 = infinities and NaNs: not graded
+            base = (sign << 31) | (e << 23)
+            m0 = int(rng.integers(0, (1 << 23) - stretch + 1))
+            firsts.append(base + m0)
+            pats.append(base + m0 + np.arange(stretch, dtype=np.int64))
+            pats.append(base + rng.integers(0, 1 << 23, scattered))
+    bits_all = np.concatenate(pats).astype(np.uint32)
+    x = torch.from_numpy(bits_all.view(np.int32).copy()).to(DEV).view(torch.float32)
+    t = table(act, 2)
+    y, _ = fb.fewbit_fwd(t, x)
+    torch.cuda.synchronize()
+    s, _ = t.arrays()
+    xn, yn = np_bits(x), np_bits(y)
+    shards = [wl.shard_range(xn.size, r, _THREADS, 1024) for r in range(_THREADS)]
+    y_ref = np.concatenate(list(_POOL.map(lambda c: oracle.fwd(act, 2, s, xn[c[0]:c[1]])[0], shards)))
+    d = ulp_distance(yn, y_ref)
+    assert d.max() <= 2, (act, int(d.max()), hex(int(bits_all[int(d.argmax())])))
+    per_group = stretch + scattered
+    in_stretch = (np.arange(xn.size) % per_group) < stretch
+    ds = d[in_stretch]
+    host_hist = [int((ds == k).sum()) for k in range(3)] + [int((ds > 2).sum())]
+    scan_hist = [0, 0, 0, 0]
+    for first in firsts:
+        r = fb.fewbit_f32_activation_scan(act, first, stretch)
+        scan_hist = [a + b for a, b in zip(scan_hist, r["hist"])]
+    assert scan_hist == host_hist, (act, scan_hist, host_hist)

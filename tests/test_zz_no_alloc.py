@@ -6,14 +6,19 @@ under a fixed budget, or they cannot risk the synchronisation an allocation
 may cause): its device staging area is a fixed array inside the library.  The
 test calls it through the C ABI twice in a row with different inputs -- the
 array keeps the first call's data, which must not leak into the second -- and
-compares every output byte with what the ordinary host entry point returns.
+compares every output byte with what the ordinary host entry point returns
+and with the oracle.  It also checks what the entry point is for: once the
+first call on the device has been made, a call changes neither the free device
+memory nor launches anything but its one kernel.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2202_00441_b200 as fb
 from paper_2202_00441_b200 import workloads as wl
+from helpers import finite_mask, ulp_distance
 
 pytestmark = pytest.mark.gpu
 
@@ -38,6 +43,31 @@ def test_static_entry_point_matches_the_workspace_entry_point_twice_in_a_row(dty
         fb.fewbit_fwd_host_static(t, x, y, p, device=dev)
         assert np.array_equal(wl.to_numpy_bits(y), wl.to_numpy_bits(y_ref)), (act, bits, n)   # same kernel: tolerance 0
         assert np.array_equal(p.numpy(), p_ref.numpy()), (act, bits, n)
+        # and against the oracle: codes bit-exact, y within 2 ulp
+        s, _ = t.arrays()
+        xn = wl.to_numpy_bits(x)
+        y_or, p_or = oracle.fwd(act, bits, s, xn)
+        assert np.array_equal(p.numpy().view(np.uint32), p_or), (act, bits, n)
+        ok = finite_mask(xn)
+        assert ulp_distance(wl.to_numpy_bits(y)[ok], y_or[ok]).max() <= 2, (act, bits, n)
+
+
+def test_static_entry_point_allocates_nothing_and_launches_one_kernel():
+    dev = torch.device("cuda", 0)
+    t = fb.fewbit_table_create("silu", 4)
+    n = 200000 + 3
+    x = torch.randn(n).bfloat16().pin_memory()
+    y = torch.empty_like(x).pin_memory()
+    p = torch.empty(fb.fewbit_packed_bytes(n, 4) // 4, dtype=torch.int32).pin_memory()
+    fb.fewbit_fwd_host_static(t, x, y, p, device=dev)        # the set-up call: loads the module that holds the array
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info(dev)
+    launches_before = fb.fewbit_launch_count()
+    for _ in range(3):
+        fb.fewbit_fwd_host_static(t, x, y, p, device=dev)
+    free_after, _ = torch.cuda.mem_get_info(dev)
+    assert free_after == free_before
+    assert fb.fewbit_launch_count() - launches_before == 3
 
 
 def test_static_entry_point_rejects_oversize_and_bad_arguments():
