@@ -195,14 +195,15 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
         use_lut = min_waves != 0 && waves >= min_waves;
     }
     if (!bf16 && prm.runs.count != 0) {
-        // binary32 (measured L2-cold at 2^20 .. 2^28 elements against the select-tree search): the 8 KB
-        // table wins at 4 bits from 2 waves for the lightest activations, from 4 for the others (8 for
-        // GELU, whose arithmetic hides the search longest); at 3 bits from 16 waves (8 for ELU and SELU),
-        // never for ReLU-like
+        // binary32 (measured L2-cold at 2^20 .. 2^28 elements against the search variants): the 8 KB
+        // table wins at 4 bits from 4 waves (8 for GELU, whose arithmetic hides the search longest, and
+        // for tanh and ELU), never for ReLU-like activations (the indexed search is as fast at any size:
+        // leaky ReLU at 2^28, 350 against 356 us); at 3 bits from 16 waves (8 for ELU and SELU), never
+        // for ReLU-like
         const int weight = act_weight(table->act);
-        const size_t min_waves4 = weight == 0 ? 2 : (table->act == FEWBIT_GELU ? 8 : 4);
+        const size_t min_waves4 = (table->act == FEWBIT_GELU || table->act == FEWBIT_TANH || table->act == FEWBIT_ELU) ? 8 : 4;
         const size_t min_waves3 = (table->act == FEWBIT_ELU || table->act == FEWBIT_SELU) ? 8 : 16;
-        use_lut = (table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && weight >= 1 && waves >= min_waves3);
+        use_lut = weight >= 1 && ((table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && waves >= min_waves3));
     }
     bool forced_table = false;
     if (const int force = option(FEWBIT_OPT_FWD_TABLE); force == 1) { use_lut = prm.runs.count != 0; forced_table = true; }
