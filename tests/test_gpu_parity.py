@@ -1057,6 +1057,57 @@ def test_stream_capture_uses_the_static_partition_and_replays():
     assert torch.equal(y2.view(torch.int16), y.view(torch.int16))
 
 
+def test_dynamic_launch_from_another_thread_while_a_capture_is_in_progress():
+    """One host thread captures a CUDA graph in the global capture mode (torch's default) while
+    another launches the dynamically distributed table variant on a stream of its own.  Leasing the
+    work counters queries CUDA events, which the global mode would refuse from any thread: the
+    library makes those calls in the relaxed mode, so the capture stays valid and both results are
+    right.  Every buffer is allocated before the capture begins (an allocation would invalidate it)."""
+    import threading
+    n = (1 << 23) + 4097
+    t = table("gelu", 4)
+    x = torch.randn(n, device=DEV).mul_(1.3).bfloat16()
+    fb.fewbit_set_option("fwd_table", "never")
+    y_ref, p_ref = fb.fewbit_fwd(t, x)
+    fb.fewbit_set_option("fwd_table", "always")
+    # use up every never-used set of work counters, so that the launch below has to query events
+    warm = [torch.cuda.Stream() for _ in range(20)]
+    for st in warm:
+        with torch.cuda.stream(st):
+            fb.fewbit_fwd(t, x)
+    torch.cuda.synchronize()
+    y_cap, p_cap = torch.zeros_like(y_ref), torch.zeros_like(p_ref)
+    y_dyn, p_dyn = torch.zeros_like(y_ref), torch.zeros_like(p_ref)
+    side = torch.cuda.Stream()
+    capturing, launched, errors = threading.Event(), threading.Event(), []
+
+    def other_thread():
+        try:
+            torch.cuda.set_device(DEV)
+            capturing.wait(timeout=60)
+            with torch.cuda.stream(side):
+                fb.fewbit_fwd(t, x, y_dyn, p_dyn)
+        except Exception as exc:                      # pragma: no cover
+            errors.append(exc)
+        finally:
+            launched.set()
+
+    th = threading.Thread(target=other_thread)
+    th.start()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        fb.fewbit_fwd(t, x, y_cap, p_cap)
+        capturing.set()
+        launched.wait(timeout=60)
+    th.join()
+    assert not errors, errors
+    graph.replay()
+    torch.cuda.synchronize()
+    for y, pk, what in ((y_cap, p_cap, "captured"), (y_dyn, p_dyn, "other thread")):
+        assert torch.equal(pk, p_ref), what
+        assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16)), what
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_graph_of_forward_and_backward_replays_with_new_inputs(dtype):
     """A captured forward -> backward chain (the backward reads the words the forward wrote, the two
