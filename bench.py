@@ -642,6 +642,7 @@ def main():
                     help="N > 1: weak = a tensor of the workload per rank; strong = one tensor cut into N shards")
     ap.add_argument("--workload", choices=sorted(wl.CONFIGS), default="c3")
     ap.add_argument("--act", default=None, help="activation of the workload to time (default: its first)")
+    ap.add_argument("--bits", default=None, help="comma-separated bit widths instead of the workload's own (profiling aid)")
     ap.add_argument("--elements", type=int, default=0,
                     help="draw only this many elements of the workload's distribution (small cases for profiling)")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -660,6 +661,8 @@ def main():
         return run_sweep(args)
     args.warmup = max(args.warmup, 0)
     case = wl.CONFIGS[args.workload]
+    if args.bits:
+        case = dataclasses.replace(case, name=f"{case.name} at bits {args.bits}", bits=tuple(int(b) for b in args.bits.split(",")))
     act = args.act or case.acts[0]
     if args.impl == "reference":
         run_reference(args, case, act)

@@ -53,8 +53,27 @@ namespace fewbit {
 #ifndef FEWBIT_LUT_STAGES_BF16
 #define FEWBIT_LUT_STAGES_BF16 1            // cp.async ring stages of the 16-bit table variant (the table takes 64 KB)
 #endif
-template <typename T, bool LUT = false> struct FwdThreads { static constexpr int value = sizeof(T) == 2 ? 512 : 384; };
+#ifndef FEWBIT_ASYNC_STAGES
+#define FEWBIT_ASYNC_STAGES 2               // cp.async ring stages of the 16-bit variants without a code table
+#endif
+// binary32 without a code table: some (activation, bits) pairs run faster as more, thinner warps --
+// compiled for 512 threads (64 registers) with a one-stage ring (4 KB of shared memory per warp), so
+// that 32 warps are resident per SM instead of 24.  (The second ring stage is never filled: these
+// variants take one warp-block per warp.)  Measured L2-cold at 2^24 and 2^28 elements, search variants:
+// 3 bits, every activation with an exponential or tanh: 5-7 % faster (sigmoid 27.1 -> 25.9 us and
+// 366 -> 346 us, softplus 28.4 -> 26.4 and 389 -> 365); 4 bits: sigmoid 33.3 -> 30.7 / 463 -> 408,
+// SiLU 33.6 -> 31.8 / 467 -> 425, softplus equal / 471 -> 454, but ELU, SELU, tanh and the ReLUs
+// 3-8 % slower (they keep 384 threads); 2 bits: SiLU only (334 -> 323 us).  GELU is bound by the FMA
+// pipe and does not change with occupancy (445 us at 1 bit with 24 or 32 warps).
+template <int ACT, int BITS>
+constexpr bool kThinWarps = (BITS == 3 && ACT != FEWBIT_LEAKY_RELU && ACT != FEWBIT_RELU) ||
+                            (BITS == 4 && (ACT == FEWBIT_SIGMOID || ACT == FEWBIT_SILU || ACT == FEWBIT_SOFTPLUS)) ||
+                            (BITS == 2 && ACT == FEWBIT_SILU);
+// (The 16-bit variants measured 1-5 % slower when compiled for 640 or 768 threads -- 40 or 48 resident warps at 48 / 40 registers.)
+template <typename T, bool LUT = false, bool THIN = false> struct FwdThreads { static constexpr int value = sizeof(T) == 2 ? 512 : ((!LUT && THIN) ? 512 : 384); };
 template <typename T, bool LUT> struct FwdCtas { static constexpr int value = 2; };
+// cp.async ring stages of the variants without a code table
+template <typename T, bool THIN> constexpr int kAsyncStages = sizeof(T) == 2 ? FEWBIT_ASYNC_STAGES : (THIN ? 1 : 2);
 
 template <typename T> constexpr bool kIsHalf = false;
 template <> constexpr bool kIsHalf<__half> = true;
@@ -136,9 +155,6 @@ __device__ __forceinline__ void add_bias(Raw<__half> &r, const __half *b, bool) 
 // ---------------------------------------------------------------------------
 #ifndef FEWBIT_INDEXED_SEARCH
 #define FEWBIT_INDEXED_SEARCH 1             // binary32 search variant at 4 bits: boundaries indexed in shared memory (0: select tree)
-#endif
-#ifndef FEWBIT_ASYNC_STAGES
-#define FEWBIT_ASYNC_STAGES 2
 #endif
 
 __device__ __forceinline__ void cp_async_chunk(uint32_t saddr, const __nv_bfloat16 *g) {
@@ -315,11 +331,11 @@ __device__ __forceinline__ uint32_t bucketize_indexed(uint32_t thr, float first,
 // FOLD: the code is the position of |x| (even f', table on [0, B]); the code tables arrive already
 // built that way, the searches strip the sign first.
 template <int ACT, int BITS, typename T, bool LUT, bool FOLD, bool BIAS = false>
-__global__ void __launch_bounds__(FwdThreads<T, LUT>::value, FwdCtas<T, LUT>::value)
+__global__ void __launch_bounds__((FwdThreads<T, LUT, kThinWarps<ACT, BITS>>::value), (FwdCtas<T, LUT>::value))
 fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters, unsigned long_ctas) {
     pdl_launch_dependents();
     constexpr bool kIsBf16 = sizeof(T) == 2;
-    constexpr int kFwdThreads = FwdThreads<T, LUT>::value;
+    constexpr int kFwdThreads = FwdThreads<T, LUT, kThinWarps<ACT, BITS>>::value;
     constexpr int kCells = kIsBf16 ? (1 << kCellBitsBf16) : (1 << kCellBitsF32);
     extern __shared__ __align__(16) uint8_t smem_raw[];
     uint8_t *lut = smem_raw;
@@ -362,7 +378,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         }
         return wb + warps;
     };
-    constexpr int kStages = LUT ? (kIsBf16 ? FEWBIT_LUT_STAGES_BF16 : 0) : FEWBIT_ASYNC_STAGES;   // 0: prefetch into registers
+    constexpr int kStages = LUT ? (kIsBf16 ? FEWBIT_LUT_STAGES_BF16 : 0) : kAsyncStages<T, kThinWarps<ACT, BITS>>;   // 0: prefetch into registers
     static_assert(kStages >= 0 && kStages <= 2, "the loop tracks two warp-blocks ahead");
     constexpr uint32_t kRingOffset = LUT ? (kCells + static_cast<uint32_t>(sizeof(FwdSmem)) + 127u) / 128u * 128u : 0u;
     constexpr uint32_t kChunkBytes = kLaneElems * sizeof(T);
@@ -604,11 +620,11 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     }
 }
 
-template <typename T, bool LUT>
+template <typename T, bool LUT, bool THIN>
 constexpr size_t fwd_smem_bytes() {
     return LUT ? ((sizeof(T) == 2 ? (1u << kCellBitsBf16) : (1u << kCellBitsF32)) + sizeof(FwdSmem) + 127u) / 128u * 128u +
                      (sizeof(T) == 2 ? static_cast<size_t>(FEWBIT_LUT_STAGES_BF16) * (FwdThreads<T, true>::value / 32) * kWarpElems * sizeof(T) : 0)
-               : static_cast<size_t>(FEWBIT_ASYNC_STAGES) * (FwdThreads<T>::value / 32) * kWarpElems * sizeof(T);
+               : static_cast<size_t>(kAsyncStages<T, THIN>) * (FwdThreads<T, false, THIN>::value / 32) * kWarpElems * sizeof(T);
 }
 
 int device_sm_count(cudaError_t *err);   // of the current device, cached
@@ -629,7 +645,8 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     cudaError_t err = cudaSuccess;
     const int sms = device_sm_count(&err);
     if (err != cudaSuccess) return err;
-    constexpr size_t smem = fwd_smem_bytes<T, LUT>();
+    constexpr bool kThin = kThinWarps<ACT, BITS>;
+    constexpr size_t smem = fwd_smem_bytes<T, LUT, kThin>();
     auto kernel = fwd_kernel<ACT, BITS, T, LUT, FOLD, BIAS>;
     if constexpr (smem > 48 * 1024) {           // opt in to the large dynamic shared memory once per device
         static std::atomic<uint64_t> opted_in{0};
@@ -643,7 +660,7 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
             opted_in.fetch_or(bit, std::memory_order_relaxed);
         }
     }
-    constexpr int kFwdThreads = FwdThreads<T, LUT>::value;
+    constexpr int kFwdThreads = FwdThreads<T, LUT, kThin>::value;
     // Without a table the CTA size is free (a warp's work does not depend on it): 4-warp CTAs fill
     // and drain the SMs more evenly than the 12 or 16 warps the kernel is compiled for (binary32
     // sigmoid, 51 M elements: 74.7 -> 70.6 us; bfloat16 SiLU, 12.6 M: 15.0 -> 12.9 us).

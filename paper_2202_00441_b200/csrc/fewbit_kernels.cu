@@ -198,12 +198,13 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
         // binary32 (measured L2-cold at 2^20 .. 2^28 elements against the search variants): the 8 KB
         // table wins at 4 bits from 4 waves (8 for GELU, whose arithmetic hides the search longest, and
         // for tanh and ELU), never for ReLU-like activations (the indexed search is as fast at any size:
-        // leaky ReLU at 2^28, 350 against 356 us); at 3 bits from 16 waves (8 for ELU and SELU), never
-        // for ReLU-like
+        // leaky ReLU at 2^28, 350 against 356 us); at 3 bits only for GELU (from 16 waves), SiLU and
+        // sigmoid (from 24: 354 against 367 us at 2^28) -- for the others the search in thin warps is
+        // as fast or faster at every size (softplus at 2^28: 364 against 377 us)
         const int weight = act_weight(table->act);
         const size_t min_waves4 = (table->act == FEWBIT_GELU || table->act == FEWBIT_TANH || table->act == FEWBIT_ELU) ? 8 : 4;
-        const size_t min_waves3 = (table->act == FEWBIT_ELU || table->act == FEWBIT_SELU) ? 8 : 16;
-        use_lut = weight >= 1 && ((table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && waves >= min_waves3));
+        const size_t min_waves3 = table->act == FEWBIT_GELU ? 16 : ((table->act == FEWBIT_SILU || table->act == FEWBIT_SIGMOID) ? 24 : 0);
+        use_lut = weight >= 1 && ((table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && min_waves3 != 0 && waves >= min_waves3));
     }
     bool forced_table = false;
     if (const int force = option(FEWBIT_OPT_FWD_TABLE); force == 1) { use_lut = prm.runs.count != 0; forced_table = true; }
