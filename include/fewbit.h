@@ -344,7 +344,11 @@ FEWBIT_API fewbit_status fewbit_fwd_host_static(const fewbit_table *table, const
  *   FEWBIT_OPT_PDL          1 programmatic dependent launch (default), 0 off;
  *   FEWBIT_OPT_COUNT_TAILS  1: every warp that runs the forward kernel's
  *                           ragged-tail path adds one to a device counter read
- *                           by fewbit_tail_warp_count (default 0: no counting).
+ *                           by fewbit_tail_warp_count (default 0: no counting);
+ *   FEWBIT_OPT_FWD_TILE     0 by size (default): small tensors are processed a
+ *                           256-element tile per warp instead of a 1024-element
+ *                           block, 1 always (variants without a code table),
+ *                           2 never.
  * fewbit_set_option returns FEWBIT_ERR_INVALID_ARG for an unknown option or a
  * value outside its range; fewbit_get_option returns -1 for an unknown option.
  */
@@ -354,7 +358,8 @@ typedef enum fewbit_option {
     FEWBIT_OPT_FWD_ITERS = 2,
     FEWBIT_OPT_FWD_WARPS = 3,
     FEWBIT_OPT_PDL = 4,
-    FEWBIT_OPT_COUNT_TAILS = 5
+    FEWBIT_OPT_COUNT_TAILS = 5,
+    FEWBIT_OPT_FWD_TILE = 6
 } fewbit_option;
 FEWBIT_API fewbit_status fewbit_set_option(fewbit_option option, int value);
 FEWBIT_API int fewbit_get_option(fewbit_option option);
@@ -362,7 +367,8 @@ FEWBIT_API int fewbit_get_option(fewbit_option option);
 /*
  * Diagnostic: *count (HOST) receives how many warps have run the ragged-tail
  * path of the forward kernel on the current device while FEWBIT_OPT_COUNT_TAILS
- * was 1 (exactly one per launch whose n is not a multiple of 1024); reset != 0
+ * was 1 (exactly one per launch whose n is not a multiple of 1024 -- of 256 for
+ * a launch in tile mode); reset != 0
  * clears the counter afterwards.  Synchronises the device.
  */
 FEWBIT_API fewbit_status fewbit_tail_warp_count(uint64_t *count, int reset);

@@ -198,13 +198,13 @@ def fewbit_launch_count() -> int:
     return int(load_library().fewbit_launch_count())
 
 
-OPTIONS = {"fwd_table": 0, "fwd_queue": 1, "fwd_iters": 2, "fwd_warps": 3, "pdl": 4, "count_tails": 5}
+OPTIONS = {"fwd_table": 0, "fwd_queue": 1, "fwd_iters": 2, "fwd_warps": 3, "pdl": 4, "count_tails": 5, "fwd_tile": 6}
 _OPTION_VALUES = {"auto": 0, "always": 1, "never": 2}
 
 
 def fewbit_set_option(option, value) -> None:
     """Process-wide testing / tuning switch; `option` by name or number, `value` an int (for
-    "fwd_table" also "auto" | "always" | "never"; for "fwd_queue" "auto" | "never")."""
+    "fwd_table" and "fwd_tile" also "auto" | "always" | "never"; for "fwd_queue" "auto" | "never")."""
     opt = OPTIONS[option] if isinstance(option, str) else int(option)
     if isinstance(value, str):
         value = {"auto": 0, "never": 1}[value] if opt == 1 else _OPTION_VALUES[value]

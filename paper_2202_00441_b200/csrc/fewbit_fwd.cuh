@@ -328,9 +328,70 @@ __device__ __forceinline__ uint32_t bucketize_indexed(uint32_t thr, float first,
     return c4;
 }
 
+// y values (o) and the 8 * BITS-bit code group of one lane-chunk: activation, interval search (whichever
+// variant the instantiation uses) and the merge of the eight codes.
+template <int ACT, int BITS, typename T, bool LUT, bool FOLD, bool kIndexed>
+__device__ __forceinline__ uint32_t chunk_codes(const Raw<T> &c, float (&o)[8], const FwdParams &prm, const uint8_t *lut, const float *thr,
+                                                uint32_t pair_table, uint32_t thr_idx) {
+    constexpr bool kIsBf16 = sizeof(T) == 2;
+    uint32_t g = 0;
+    [[maybe_unused]] uint32_t dense = 0;
+    [[maybe_unused]] uint32_t pc[4];                        // bfloat16: codes of element pair i, low @0, high @16
+#pragma unroll
+    for (int e = 6; e >= 0; e -= 2) {                       // two neighbouring elements at a time
+        const float2 xv = make_float2(elem(c, e), elem(c, e + 1));
+        const float2 yv = activation2<ACT, T>(xv);
+        o[e] = yv.x;
+        o[e + 1] = yv.y;
+        if constexpr (kIsBf16) {
+            if constexpr (LUT) {
+                pc[e / 2] = lut[cell(c, e)] + (static_cast<uint32_t>(lut[cell(c, e + 1)]) << 16);
+            } else {
+                pc[e / 2] = bucketize_bf16x2<BITS, T>(prm.sb2, FOLD ? (pair_bits(c, e) & 0x7fff7fffu) : pair_bits(c, e), pair_table);
+            }
+        } else {
+            uint32_t c0, c1;
+            const float k0 = FOLD ? fabsf(xv.x) : xv.x, k1 = FOLD ? fabsf(xv.y) : xv.y;   // what is searched for
+            if constexpr (kIndexed) {
+                const float mid = prm.tb.s[(1 << (BITS - 1)) - 1];
+                c0 = bucketize_indexed<BITS>(thr_idx, mid, k0);
+                c1 = bucketize_indexed<BITS>(thr_idx, mid, k1);
+                c0 = ((c1 << BITS) + c0) >> 2;              // both codes at once: (c1 << BITS) + c0
+                c1 = 0;
+            } else if constexpr (!LUT) {
+                c0 = bucketize<BITS>(prm.tb, k0);
+                c1 = bucketize<BITS>(prm.tb, k1);
+            } else {
+                const uint32_t m0 = lut[cell(c, e)], m1 = lut[cell(c, e + 1)];
+                dense |= m0 | m1;
+                c0 = (m0 & 15u) + (thr[m0 & 15u] < k0 ? 1u : 0u);
+                c1 = (m1 & 15u) + (thr[m1 & 15u] < k1 ? 1u : 0u);
+            }
+            g = kIndexed ? (g << (2 * BITS)) + c0 : (((g << BITS) + c1) << BITS) + c0;
+        }
+    }
+    if constexpr (kIsBf16) {
+        // eight codes -> one 8*BITS-bit group: merge pairs two by two while the low and the
+        // high elements still sit in separate halves, then fold the high half next to the low
+        const uint32_t a01 = pc[0] + (pc[1] << (2 * BITS)), a23 = pc[2] + (pc[3] << (2 * BITS));
+        constexpr uint32_t kFold = (1u << BITS) - (1u << 16);               // hi * 2^16 -> hi * 2^BITS
+        const uint32_t b01 = a01 + (a01 >> 16) * kFold, b23 = a23 + (a23 >> 16) * kFold;
+        g = b01 + (b23 << (4 * BITS));
+    }
+    if constexpr (LUT && !kIsBf16) {
+        if (__any_sync(0xffffffffu, dense & 0x80u)) {        // a dense cell: redo this tile's codes by search
+            g = 0;
+#pragma unroll
+            for (int e = 7; e >= 0; --e)
+                g = (g << BITS) + bucketize<BITS>(prm.tb, FOLD ? fabsf(elem(c, e)) : elem(c, e));
+        }
+    }
+    return g;
+}
+
 // FOLD: the code is the position of |x| (even f', table on [0, B]); the code tables arrive already
 // built that way, the searches strip the sign first.
-template <int ACT, int BITS, typename T, bool LUT, bool FOLD, bool BIAS = false>
+template <int ACT, int BITS, typename T, bool LUT, bool FOLD, bool BIAS = false, bool TILE = false>
 __global__ void __launch_bounds__((FwdThreads<T, LUT, kThinWarps<ACT, BITS>>::value), (FwdCtas<T, LUT>::value))
 fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *packed, size_t n, int iters, unsigned long_ctas) {
     pdl_launch_dependents();
@@ -418,6 +479,54 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         thr_idx = static_cast<uint32_t>(__cvta_generic_to_shared(thr_s));
     }
     pdl_wait();                                                     // nothing above touches global memory
+    // Tile mode (small tensors, variants without a code table): one 256-element tile per warp instead
+    // of a 1024-element warp-block, so that a tensor of a few hundred thousand elements still puts
+    // several warps on every scheduler.  The four lanes of a quad hold 32 consecutive codes between
+    // them: each lane fetches the other three groups by shuffle, assembles the BITS words and lane r
+    // of the quad stores word r.  Same bit stream as the warp-block path.
+    // A separate instantiation (TILE), so that the warp-block path compiles exactly as without it.
+    [[maybe_unused]] size_t tile_tail_begin = 0;                    // tile mode: first element of the ragged tail
+    [[maybe_unused]] bool tile_tail_owner = false;
+    if constexpr (TILE) {
+        static_assert(!LUT, "tile mode has no code table");
+        {
+            const size_t tile = static_cast<size_t>(blockIdx.x) * warps + (threadIdx.x >> 5);
+            const size_t full_tiles = n / kTileElems;
+            if (tile < full_tiles) {
+                const size_t base = tile * kTileElems + static_cast<size_t>(lane) * kLaneElems;
+                Raw<T> c;
+                load_raw(x + base, c, wide);
+                if constexpr (BIAS) {
+                    const uint64_t chunk = tile * 32;                        // number of the tile's first lane-chunk
+                    const uint32_t row_chunks = prm.cols / kLaneElems;
+                    const uint64_t rem = chunk < (1ull << 32) ? chunk - __umul64hi(chunk, prm.chunks_magic) * row_chunks : chunk % row_chunks;
+                    uint64_t col = (rem + lane) * kLaneElems;
+                    if (col >= prm.cols) col = prm.cols >= kTileElems ? col - prm.cols : col % prm.cols;
+                    add_bias(c, static_cast<const T *>(prm.bias) + col, wide);
+                }
+                float o[8];
+                const uint32_t g = chunk_codes<ACT, BITS, T, LUT, FOLD, kIndexed>(c, o, prm, lut, thr, pair_table, thr_idx);
+                store8(y + base, o, wide);
+                uint32_t grp[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) grp[j] = __shfl_sync(0xffffffffu, g, (lane & ~3) + j);
+                uint32_t w[BITS];
+                groups_to_words<BITS>(grp, w);
+                const int r = lane & 3;
+                if (r < BITS) {
+                    uint32_t word = w[0];
+#pragma unroll
+                    for (int j = 1; j < BITS; ++j) word = r == j ? w[j] : word;
+                    packed[tile * (8 * BITS) + (lane >> 2) * BITS + r] = word;
+                }
+                return;
+            }
+            tile_tail_begin = full_tiles * kTileElems;
+            tile_tail_owner = tile == full_tiles;
+            if (!tile_tail_owner) return;
+        }
+    }
+    if constexpr (!TILE) {                                          // (in tile mode only the tail's owner gets here, and skips to the tail)
     Raw<T> cur[kTilesPerWarp];
     size_t wb = first_wb;                                           // the warp-block in hand, the one after it,
     size_t nxt = wb < full ? next_after(wb) : full;                 // and (inside the loop) the one after that
@@ -478,58 +587,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
                 }
             }
             float o[8];
-            uint32_t g = 0;
-            [[maybe_unused]] uint32_t dense = 0;
-            [[maybe_unused]] uint32_t pc[4];                        // bfloat16: codes of element pair i, low @0, high @16
-#pragma unroll
-            for (int e = 6; e >= 0; e -= 2) {                       // two neighbouring elements at a time
-                const float2 xv = make_float2(elem(cur[t], e), elem(cur[t], e + 1));
-                const float2 yv = activation2<ACT, T>(xv);
-                o[e] = yv.x;
-                o[e + 1] = yv.y;
-                if constexpr (kIsBf16) {
-                    if constexpr (LUT) {
-                        pc[e / 2] = lut[cell(cur[t], e)] + (static_cast<uint32_t>(lut[cell(cur[t], e + 1)]) << 16);
-                    } else {
-                        pc[e / 2] = bucketize_bf16x2<BITS, T>(prm.sb2, FOLD ? (pair_bits(cur[t], e) & 0x7fff7fffu) : pair_bits(cur[t], e), pair_table);
-                    }
-                } else {
-                    uint32_t c0, c1;
-                    const float k0 = FOLD ? fabsf(xv.x) : xv.x, k1 = FOLD ? fabsf(xv.y) : xv.y;   // what is searched for
-                    if constexpr (kIndexed) {
-                        const float mid = prm.tb.s[(1 << (BITS - 1)) - 1];
-                        c0 = bucketize_indexed<BITS>(thr_idx, mid, k0);
-                        c1 = bucketize_indexed<BITS>(thr_idx, mid, k1);
-                        c0 = ((c1 << BITS) + c0) >> 2;              // both codes at once: (c1 << BITS) + c0
-                        c1 = 0;
-                    } else if constexpr (!LUT) {
-                        c0 = bucketize<BITS>(prm.tb, k0);
-                        c1 = bucketize<BITS>(prm.tb, k1);
-                    } else {
-                        const uint32_t m0 = lut[cell(cur[t], e)], m1 = lut[cell(cur[t], e + 1)];
-                        dense |= m0 | m1;
-                        c0 = (m0 & 15u) + (thr[m0 & 15u] < k0 ? 1u : 0u);
-                        c1 = (m1 & 15u) + (thr[m1 & 15u] < k1 ? 1u : 0u);
-                    }
-                    g = kIndexed ? (g << (2 * BITS)) + c0 : (((g << BITS) + c1) << BITS) + c0;
-                }
-            }
-            if constexpr (kIsBf16) {
-                // eight codes -> one 8*BITS-bit group: merge pairs two by two while the low and the
-                // high elements still sit in separate halves, then fold the high half next to the low
-                const uint32_t a01 = pc[0] + (pc[1] << (2 * BITS)), a23 = pc[2] + (pc[3] << (2 * BITS));
-                constexpr uint32_t kFold = (1u << BITS) - (1u << 16);               // hi * 2^16 -> hi * 2^BITS
-                const uint32_t b01 = a01 + (a01 >> 16) * kFold, b23 = a23 + (a23 >> 16) * kFold;
-                g = b01 + (b23 << (4 * BITS));
-            }
-            if constexpr (LUT && !kIsBf16) {
-                if (__any_sync(0xffffffffu, dense & 0x80u)) {        // a dense cell: redo this tile's codes by search
-                    g = 0;
-#pragma unroll
-                    for (int e = 7; e >= 0; --e)
-                        g = (g << BITS) + bucketize<BITS>(prm.tb, FOLD ? fabsf(elem(cur[t], e)) : elem(cur[t], e));
-                }
-            }
+            const uint32_t g = chunk_codes<ACT, BITS, T, LUT, FOLD, kIndexed>(cur[t], o, prm, lut, thr, pair_table, thr_idx);
             grp[t] = g;
             store8(py + t * kTileElems, o, wide);
             if constexpr (kStages == 0) {
@@ -554,16 +612,17 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
         wb = nxt;
         nxt = nxt2;
     }
+    }
 
     // ragged tail: the one warp whose sequence warp0, warp0 + warps, ... reaches the index of the last,
     // partial warp-block (all_full >= warp0 keeps the unsigned difference from wrapping: 2^64 is not a
     // multiple of every CTA width); a lane owns 32 consecutive elements = BITS words
-    const bool owns_tail = dynamic ? (blockIdx.x == 0 && threadIdx.x < 32)
+    const bool owns_tail = TILE ? true : dynamic ? (blockIdx.x == 0 && threadIdx.x < 32)
                                    : (all_full >= warp0 && all_full < cta_end && (all_full - warp0) % warps == 0);
-    if ((n % kWarpElems) != 0 && owns_tail) {
+    const size_t tail_begin = TILE ? tile_tail_begin : all_full * kWarpElems;   // first element of the ragged tail
+    if ((TILE ? tail_begin != n : (n % kWarpElems) != 0) && owns_tail) {
         if (prm.tail_counter != nullptr && lane == 0) atomicAdd(prm.tail_counter, 1u);
-        const size_t full = all_full;
-        const size_t base = full * kWarpElems + static_cast<size_t>(lane) * 32;
+        const size_t base = tail_begin + static_cast<size_t>(lane) * 32;
         uint32_t w[BITS + 1];
 #pragma unroll
         for (int j = 0; j <= BITS; ++j) w[j] = 0;
@@ -596,7 +655,7 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
             }
         }
         const size_t total_words = (n * BITS + 31) / 32;
-        const size_t first = full * (32 * BITS) + static_cast<size_t>(lane) * BITS;
+        const size_t first = (TILE ? tail_begin / 32 * BITS : all_full * (32 * BITS)) + static_cast<size_t>(lane) * BITS;
 #pragma unroll
         for (int j = 0; j < BITS; ++j)
             if (first + j < total_words) packed[first + j] = w[j];
@@ -635,10 +694,19 @@ constexpr int act_weight(int act) {
     return (act == FEWBIT_RELU || act == FEWBIT_LEAKY_RELU) ? 0
          : (act == FEWBIT_GELU || act == FEWBIT_SILU) ? 2 : 1;
 }
+// Tile mode below this many warp-blocks per resident warp (numerator / denominator), measured L2-cold
+// in batches of 8 launches, tile mode against warp-blocks: binary32 at 2^20 elements GELU 3 bits
+// 6.4 -> 5.1 us, SiLU 4 bits 6.1 -> 4.4; at 2^21 10.0 -> 7.4 and 9.2 -> 6.4; 2^14 .. 2^19: 3.6-4.9 ->
+// 2.3-4.1; from 2^22 (one wave) on equal or slower.  16-bit types: 2^20 4.0-4.4 -> 3.3-3.6 us, 2^21
+// 5.6-6.1 -> 4.9-5.1 (the cheapest, 1-bit leaky ReLU: 3.8 -> 4.4), 2^22 (0.86 waves) 6.1-7.7 -> 6.7-8.7:
+// hence one half.
+template <typename T> constexpr size_t kTileModeNum = 1;
+template <typename T> constexpr size_t kTileModeDen = sizeof(T) == 2 ? 2 : 1;
 constexpr size_t kLutMinIters = 8;      // below this many warp-blocks per warp the table does not pay for its expansion
 int fwd_iters_override();                // FEWBIT_OPT_FWD_ITERS: 0 = the size-based choice
 bool pdl_enabled();                      // FEWBIT_OPT_PDL
 int fwd_warps_override();                // FEWBIT_OPT_FWD_WARPS (variants without a table): 0 = the default
+int fwd_tile_mode();                     // FEWBIT_OPT_FWD_TILE: 0 = by size, 1 = tile mode whenever there is no table, 2 = never
 
 template <int ACT, int BITS, typename T, bool LUT, bool FOLD, bool BIAS = false>
 cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *packed, size_t n, cudaStream_t st) {
@@ -725,6 +793,18 @@ cudaError_t launch_fwd(const FwdParams &prm, const void *x, void *y, uint32_t *p
     // tensors go from 4.2 us to ~2 us apiece, and no size or activation measured slower with it
     // (batches of 8 launches, 2^16 .. 2^28 elements).
     const bool pdl = pdl_enabled();
+    if constexpr (!LUT) {
+        // Tile mode for small tensors: with fewer warp-blocks than a fraction of the resident warps, a
+        // 256-element tile per warp puts four times as many warps to work (measurements at kTileModeNum).
+        const int mode = fwd_tile_mode();
+        const size_t resident_warps = slots * warps_per_cta;
+        if (mode == 1 || (mode == 0 && warp_blocks * kTileModeDen<T> < resident_warps * kTileModeNum<T>)) {
+            const size_t tiles = n / kTileElems + ((n % kTileElems) ? 1 : 0);
+            const unsigned tgrid = static_cast<unsigned>((tiles + warps_per_cta - 1) / warps_per_cta);
+            return launch_pdl(fwd_kernel<ACT, BITS, T, false, FOLD, BIAS, true>, tgrid, static_cast<unsigned>(warps_per_cta * 32), 0, st, pdl,
+                              p2, static_cast<const T *>(x), static_cast<T *>(y), packed, n, 1, tgrid);
+        }
+    }
     return launch_pdl(kernel, grid, static_cast<unsigned>(warps_per_cta * 32), smem * warps_per_cta / (kFwdThreads / 32), st, pdl,
                       p2, static_cast<const T *>(x), static_cast<T *>(y), packed, n, static_cast<int>(iters), n_long);
 }

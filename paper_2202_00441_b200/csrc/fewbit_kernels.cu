@@ -128,13 +128,14 @@ int device_sm_count(cudaError_t *err) {
 
 // Process-wide options (fewbit_set_option): plain atomics, read with relaxed loads on every launch.
 // No environment variable is read anywhere in the library.
-constexpr int kNumOptions = 6;
-std::atomic<int> g_option[kNumOptions] = {{0}, {0}, {0}, {0}, {1}, {0}};   // defaults; FEWBIT_OPT_PDL is on
+constexpr int kNumOptions = 7;
+std::atomic<int> g_option[kNumOptions] = {{0}, {0}, {0}, {0}, {1}, {0}, {0}};   // defaults; FEWBIT_OPT_PDL is on
 inline int option(fewbit_option o) { return g_option[o].load(std::memory_order_relaxed); }
 
 int fwd_iters_override() { return option(FEWBIT_OPT_FWD_ITERS); }
 bool pdl_enabled() { return option(FEWBIT_OPT_PDL) != 0; }
 int fwd_warps_override() { return option(FEWBIT_OPT_FWD_WARPS); }
+int fwd_tile_mode() { return option(FEWBIT_OPT_FWD_TILE); }
 
 inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -290,6 +291,7 @@ fewbit_status fewbit_set_option(fewbit_option opt, int value) {
     case FEWBIT_OPT_FWD_WARPS: ok = value >= 0 && value <= 16; break;
     case FEWBIT_OPT_PDL: ok = value == 0 || value == 1; break;
     case FEWBIT_OPT_COUNT_TAILS: ok = value == 0 || value == 1; break;
+    case FEWBIT_OPT_FWD_TILE: ok = value >= 0 && value <= 2; break;
     default: break;
     }
     if (!ok) return FEWBIT_ERR_INVALID_ARG;

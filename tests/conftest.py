@@ -35,5 +35,5 @@ def _default_library_options():
     except Exception:  # pragma: no cover
         return
     if binding._lib is not None:
-        for opt, default in ((0, 0), (1, 0), (2, 0), (3, 0), (4, 1), (5, 0)):
+        for opt, default in ((0, 0), (1, 0), (2, 0), (3, 0), (4, 1), (5, 0), (6, 0)):
             binding._lib.fewbit_set_option(opt, default)

@@ -927,6 +927,57 @@ def test_ragged_tail_has_one_owner_and_works_in_place(dtype, bits):
             assert torch.equal(pb, p0) and torch.equal(yb.view(torch.uint8).reshape(-1), y0.view(torch.uint8).reshape(-1))
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+def test_tile_mode_gives_the_same_stream(dtype, bits):
+    """Small tensors are processed a 256-element tile per warp (the quad of lanes assembles the words
+    by shuffle) instead of a 1024-element warp-block.  Forced on at every size class -- ragged below
+    one tile, whole tiles, tails at every 32-element offset of a tile, a few hundred tiles -- it gives
+    the oracle's codes and grad_in and y within 2 ulp, the bytes of the warp-block path, in place as
+    well, with the bias in front as well, and exactly one warp runs the ragged tail."""
+    tdt = TORCH_DT[dtype]
+    gen = torch.Generator(device=DEV).manual_seed(29 + bits)
+    fb.fewbit_set_option("count_tails", 1)
+    fb.fewbit_tail_warp_count(reset=True)
+    sizes = [1, 31, 32, 33, 255, 256, 257, 511, 1023, 1024, 1025, 2048 + 33, 9999, 70001, (1 << 18) + 256 * 3]
+    sizes += [256 * 5 + 32 * k + 3 for k in range(8)]
+    for act in ("gelu", "tanh"):
+        t = table(act, bits)
+        for n in sizes:
+            x = (torch.randn(n, generator=gen, device=DEV) * 2).to(tdt)
+            g = torch.randn(n, generator=gen, device=DEV).to(tdt)
+            fb.fewbit_set_option("fwd_tile", "never")
+            y0, p0 = fb.fewbit_fwd(t, x)
+            fb.fewbit_tail_warp_count(reset=True)
+            fb.fewbit_set_option("fwd_tile", "always")
+            words = fb.fewbit_packed_bytes(n, bits) // 4
+            pbuf, pk, ppad = guarded(words, torch.int32, 0x5A5A5A5A)
+            ybuf, y, ypad = guarded(n, tdt, 777.0)
+            fb.fewbit_fwd(t, x, y, pk)
+            assert fb.fewbit_tail_warp_count(reset=True) == (1 if n % 256 else 0), (dtype, bits, act, n)
+            check_guards(ybuf, n, ypad, 777.0)
+            check_guards(pbuf, words, ppad, 0x5A5A5A5A)
+            assert torch.equal(pk, p0) and torch.equal(y.view(torch.uint8), y0.view(torch.uint8)), (dtype, bits, act, n)
+            xi = x.clone()
+            pi = torch.empty_like(p0)
+            fb.fewbit_fwd(t, xi, xi, pi)                                  # in place
+            assert torch.equal(pi, p0) and torch.equal(xi.view(torch.uint8), y0.view(torch.uint8)), (dtype, bits, act, n)
+            if n <= 70001:
+                gi = fb.fewbit_bwd(t, pk, g)
+                compare_full(act, bits, x, g, y, pk, gi, f"tile mode {dtype} k={bits} {act} n={n}")
+            for cols in (8, 200, 1024):                                   # rows shorter than, straddling and longer than a tile
+                rows = n // cols
+                if rows:
+                    m = rows * cols
+                    bias = torch.randn(cols, generator=gen, device=DEV).to(tdt)
+                    fb.fewbit_set_option("fwd_tile", "never")
+                    yb0, pb0 = fb.fewbit_fwd_bias(t, x[:m].view(rows, cols), bias)
+                    fb.fewbit_set_option("fwd_tile", "always")
+                    yb1, pb1 = fb.fewbit_fwd_bias(t, x[:m].view(rows, cols), bias)
+                    assert torch.equal(pb0, pb1) and torch.equal(yb0.view(torch.uint8), yb1.view(torch.uint8)), (dtype, bits, act, n, cols)
+    fb.fewbit_tail_warp_count(reset=True)
+
+
 @pytest.mark.parametrize("warps,iters", [(1, 0), (2, 5), (0, 1), (0, 64), (16, 2), (3, 0)])
 def test_launch_geometry_overrides_do_not_change_the_result(warps, iters):
     """FEWBIT_OPT_FWD_WARPS / FEWBIT_OPT_FWD_ITERS only reshape the grid (a single-warp CTA included):

@@ -150,7 +150,7 @@ def test_hot_path_argument_checks_need_no_gpu(lib):
     assert lib.fewbit_set_option(99, 0) == 1 and lib.fewbit_get_option(99) == -1
     assert lib.fewbit_set_option(0, 3) == 1 and lib.fewbit_set_option(2, -1) == 1 and lib.fewbit_set_option(2, 65) == 1
     assert lib.fewbit_set_option(3, 17) == 1 and lib.fewbit_set_option(4, 2) == 1
-    for opt, default, other in ((0, 0, 2), (1, 0, 1), (2, 0, 7), (3, 0, 4), (4, 1, 0), (5, 0, 1)):
+    for opt, default, other in ((0, 0, 2), (1, 0, 1), (2, 0, 7), (3, 0, 4), (4, 1, 0), (5, 0, 1), (6, 0, 2)):
         assert lib.fewbit_get_option(opt) == default
         assert lib.fewbit_set_option(opt, other) == 0 and lib.fewbit_get_option(opt) == other
         assert lib.fewbit_set_option(opt, default) == 0
