@@ -142,8 +142,11 @@ def dist_setup(n_gpus: int):
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        os.environ.setdefault("NCCL_DEBUG", "INFO")          # the communicator log shows the rank count
+        # the communicator log shows the rank count; it goes to a file per process, never to stdout
+        # (stdout carries the one JSON line)
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
         os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        os.environ.setdefault("NCCL_DEBUG_FILE", os.path.join(tempfile.gettempdir(), "fewbit_bench_nccl_%h_%p.log"))
         torch.cuda.set_device(local)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     return rank, world, local
@@ -453,7 +456,7 @@ def run_ours(args, case: wl.Case, act: str):
                        "elements_counted": "once per kernel pass (forward and backward each count n)",
                        "parallelism": (f"one tensor cut into {world} shards on multiples of 32 elements" if strong
                                        else f"independent tensors x{world}") + ", no collective on the data path"},
-            "checksum": checksum,
+            "checksum": checksum, "nccl_log": os.environ.get("NCCL_DEBUG_FILE") if world > 1 else None,
             "hbm_gbs": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9,
             "hbm_frac_of_nominal_8TBs": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS / world,
             "hbm_frac_of_measured_copy": bytes_per_step * args.steps / (total_ms * 1e-3) / 1e9 / peak / world,
