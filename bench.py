@@ -474,9 +474,9 @@ def run_ours(args, case: wl.Case, act: str):
 # captures of the 2^27-element launches of these kernels; None for a kernel without a capture.
 NCU_TRAFFIC_BYTES_PER_ELEM = {
     # scaled per element: a lower bound for the full launch, the L2 keeps ~55 MB of dirty lines either way
-    ("bf16", "fwd_k4"): 4.097,
-    ("bf16", "bwd_k4"): 4.101,
-    ("bf16", "fwd_k1"): 3.731,
+    ("bf16", "fwd_k4"): 4.098,
+    ("bf16", "bwd_k4"): 4.085,
+    ("bf16", "fwd_k1"): 3.729,
 }
 
 
