@@ -199,7 +199,9 @@ FEWBIT_API size_t fewbit_packed_bytes(size_t n, int bits);
  * first such call on a device creates up to 16 CUDA events, and each call
  * records one after its kernel).  While `stream` is being captured,
  * or when all sets are in use by other streams, the kernel falls back to a
- * static partition: same results, ~10 % slower.  The choices can be overridden
+ * static partition: same results, ~10 % slower.  Small tensors (fewer 1024-
+ * element blocks than resident warps) are processed a 256-element tile per
+ * warp, which puts four times as many warps to work.  The choices can be overridden
  * for testing and tuning with fewbit_set_option (below); the library reads no
  * environment variable.
  * Both device kernels are launched with programmatic stream serialization:
