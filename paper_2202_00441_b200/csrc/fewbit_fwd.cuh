@@ -313,7 +313,10 @@ __device__ __forceinline__ uint32_t bucketize_bf16x2(const uint32_t (&S)[kMaxLev
 // against the select tree (L2-cold, 2^22 .. 2^28 elements): 4 bits, tanh 30.7 -> 28.0 us and leaky
 // ReLU 27.9 -> 25.2 us at 2^24, 420 -> 394 and 384 -> 350 us at 2^28, SiLU equal; slower at 3 bits
 // (the tree is 4 selects there) and for GELU, whose arithmetic leaves the ALU pipe that runs the
-// selects idle anyway (39.9 -> 42.8 us): used at 4 bits for every activation but GELU.
+// selects idle anyway (39.9 -> 42.8 us): used at 4 bits for every activation but GELU.  Each warp
+// keeps its own copy of the 16 words, written by the warp itself: a CTA-wide barrier in front of a
+// CTA that lives for one warp-block per warp cost 6-10 % (tanh at 2^24: 28.0 -> 26.1 us, leaky ReLU
+// 25.0 -> 23.6, sigmoid at 2^23: 18.2 -> 16.4).
 // Returns 4 * code (the running byte offset); `first` is the middle boundary.
 // ---------------------------------------------------------------------------
 template <int BITS>
@@ -463,20 +466,24 @@ fwd_kernel(const __grid_constant__ FwdParams prm, const T *x, T *y, uint32_t *pa
     // prefixes (low element * 8 + high element), 64 words
     [[maybe_unused]] uint32_t pair_table = 0;
     if constexpr (kIsBf16 && !LUT && BITS == 4) {
-        __shared__ uint32_t last_pair[64];
-        for (uint32_t i = threadIdx.x; i < 64; i += blockDim.x)           // a CTA may be a single warp
-            last_pair[i] = (prm.sb2[2 * (i >> 3)] & 0x0000ffffu) | (prm.sb2[2 * (i & 7)] & 0xffff0000u);
-        __syncthreads();
-        pair_table = static_cast<uint32_t>(__cvta_generic_to_shared(last_pair));
+        // one copy per warp, filled by the warp itself: no CTA-wide barrier at the start of these short-lived CTAs
+        __shared__ uint32_t last_pair[kFwdThreads / 32][64];
+        uint32_t *mine = last_pair[threadIdx.x >> 5];
+#pragma unroll
+        for (uint32_t i = lane; i < 64; i += 32)
+            mine[i] = (prm.sb2[2 * (i >> 3)] & 0x0000ffffu) | (prm.sb2[2 * (i & 7)] & 0xffff0000u);
+        __syncwarp();
+        pair_table = static_cast<uint32_t>(__cvta_generic_to_shared(mine));
     }
     // binary32 without a code table, 4 bits: the boundaries in shared memory for the indexed search
     constexpr bool kIndexed = FEWBIT_INDEXED_SEARCH && !kIsBf16 && !LUT && BITS == 4 && ACT != FEWBIT_GELU;
     [[maybe_unused]] uint32_t thr_idx = 0;
     if constexpr (kIndexed) {
-        __shared__ float thr_s[kMaxLevels];
-        if (threadIdx.x < kMaxLevels) thr_s[threadIdx.x] = prm.tb.s[threadIdx.x];
-        __syncthreads();
-        thr_idx = static_cast<uint32_t>(__cvta_generic_to_shared(thr_s));
+        __shared__ float thr_s[kFwdThreads / 32][kMaxLevels];       // one copy per warp: no CTA-wide barrier
+        float *mine = thr_s[threadIdx.x >> 5];
+        if (lane < kMaxLevels) mine[lane] = prm.tb.s[lane];
+        __syncwarp();
+        thr_idx = static_cast<uint32_t>(__cvta_generic_to_shared(mine));
     }
     pdl_wait();                                                     // nothing above touches global memory
     // Tile mode (small tensors, variants without a code table): one 256-element tile per warp instead

@@ -196,16 +196,18 @@ fewbit_status forward(const fewbit_table *table, const void *x, const void *bias
         use_lut = min_waves != 0 && waves >= min_waves;
     }
     if (!bf16 && prm.runs.count != 0) {
-        // binary32 (measured L2-cold at 2^20 .. 2^28 elements against the search variants): the 8 KB
-        // table wins at 4 bits from 4 waves (8 for GELU, whose arithmetic hides the search longest, and
-        // for tanh and ELU), never for ReLU-like activations (the indexed search is as fast at any size:
-        // leaky ReLU at 2^28, 350 against 356 us); at 3 bits only for GELU (from 16 waves), SiLU and
-        // sigmoid (from 24: 354 against 367 us at 2^28) -- for the others the search in thin warps is
-        // as fast or faster at every size (softplus at 2^28: 364 against 377 us)
-        const int weight = act_weight(table->act);
-        const size_t min_waves4 = (table->act == FEWBIT_GELU || table->act == FEWBIT_TANH || table->act == FEWBIT_ELU) ? 8 : 4;
-        const size_t min_waves3 = table->act == FEWBIT_GELU ? 16 : ((table->act == FEWBIT_SILU || table->act == FEWBIT_SIGMOID) ? 24 : 0);
-        use_lut = weight >= 1 && ((table->bits == 4 && waves >= min_waves4) || (table->bits == 3 && min_waves3 != 0 && waves >= min_waves3));
+        // binary32 (measured L2-cold at 2^20 .. 2^28 elements against the search variants): at 4 bits the
+        // 8 KB table wins from 8 waves for GELU, SiLU, sigmoid and softplus (SiLU at 2^28: 361 against 415
+        // us; at 2^24, 4.6 waves, 32.2 against 30.0), from 16 for tanh (2^26: 94 against 96 us), never for
+        // ELU, SELU and the ReLU-like activations, where the indexed search is faster at every size (ELU at
+        // 2^28: 337 against 349 us); at 3 bits only for GELU (from 16 waves), SiLU and sigmoid (from 24: 354
+        // against 367 us at 2^28) -- for the others the search in thin warps is as fast or faster at every
+        // size (softplus at 2^28: 364 against 377 us)
+        const int a = table->act;
+        const size_t min_waves4 = (a == FEWBIT_GELU || a == FEWBIT_SILU || a == FEWBIT_SIGMOID || a == FEWBIT_SOFTPLUS) ? 8
+                                : (a == FEWBIT_TANH ? 16 : 0);
+        const size_t min_waves3 = a == FEWBIT_GELU ? 16 : ((a == FEWBIT_SILU || a == FEWBIT_SIGMOID) ? 24 : 0);
+        use_lut = (table->bits == 4 && min_waves4 != 0 && waves >= min_waves4) || (table->bits == 3 && min_waves3 != 0 && waves >= min_waves3);
     }
     bool forced_table = false;
     if (const int force = option(FEWBIT_OPT_FWD_TABLE); force == 1) { use_lut = prm.runs.count != 0; forced_table = true; }
