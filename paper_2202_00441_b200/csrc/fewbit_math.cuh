@@ -167,8 +167,9 @@ __device__ __forceinline__ float act_f64(float xf) {
 // every result that uses it has reached its limit in binary32 by then).  Cody-Waite reduction by
 // ln 2 in two pieces, degree-6 polynomial (fit in fit_coefficients.py: 0.05 ulp).  Returns s; *t
 // holds 1.5 * 2^23 + n, i.e. the integer n in its low mantissa bits.
+template <bool CLAMP = true>                 // CLAMP = false: the caller has already bounded a from below
 __device__ __forceinline__ float2 exp_reduced_f32(float2 a, float2 *t_out) {
-    a = make_float2(fmaxf(a.x, -131.0f), fmaxf(a.y, -131.0f));
+    if constexpr (CLAMP) a = make_float2(fmaxf(a.x, -131.0f), fmaxf(a.y, -131.0f));
     const float2 t = fma2(a, splat(kLog2e), splat(12582912.0f));
     const float2 n = add2(t, splat(-12582912.0f));
     float2 r = fma2(n, splat(-0.693145751953125f), a);                      // ln 2, high 12 bits
@@ -199,7 +200,7 @@ __device__ __forceinline__ float2 exp_scaled_f32(float2 a) {
 __device__ __forceinline__ float2 expm1_nonpos_f32(float2 a) {
     a = make_float2(fmaxf(a.x, -80.0f), fmaxf(a.y, -80.0f));
     float2 t;
-    const float2 s = exp_reduced_f32(a, &t);
+    const float2 s = exp_reduced_f32<false>(a, &t);
     const float2 p2 = pow2_from_t(t, 127u);
     return fma2(p2, s, add2(p2, splat(-1.0f)));
 }
